@@ -1,0 +1,191 @@
+"""CPU oracle for the block-rotated MXFP4 linear layer — TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper over ``bro_ref.c`` (plain C, fp32 rotation in a fixed operation order, fp64
+GEMM).  Only the tests, the smoke check and the benchmark's CPU-baseline leg import this
+package; the CUDA library never does, and the two share no code.
+
+All arrays are numpy: bf16 tensors are passed as ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libbro_ref.so")
+_SRC = [os.path.join(_HERE, "bro_ref.c")]
+_HDR = [os.path.join(_HERE, "bro_ref.h")]
+_lib = None
+
+MX_GROUP = 32
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    newest = max(os.path.getmtime(p) for p in _SRC + _HDR)
+    if not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= newest:
+        return _SO
+    cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+           "-shared", "-fPIC", "-Wall", "-Wextra", "-o", _SO] + _SRC + ["-lm"]
+    subprocess.run(cmd, check=True)
+    return _SO
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_SO)
+        i64, p, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        L.bro_ref_num_threads.restype = ci
+        L.bro_ref_set_num_threads.argtypes = [ci]
+        L.bro_ref_hadamard_norm.restype = ctypes.c_float
+        L.bro_ref_hadamard_norm.argtypes = [i64]
+        L.bro_ref_rotate.argtypes = [p, i64, i64, i64, ci, p]
+        L.bro_ref_quantize.argtypes = [p, i64, i64, p, p]
+        L.bro_ref_decode.argtypes = [p, p, i64, i64, p]
+        L.bro_ref_rotate_quantize_mxfp4.argtypes = [p, i64, i64, i64, ci, p, p]
+        L.bro_ref_pack_weights.argtypes = [p, i64, i64, i64, ci, p, p]
+        L.bro_ref_gemm_mxfp4.argtypes = [p, p, p, p, i64, i64, i64, p, p]
+        L.bro_ref_gemm_mxfp4_points.argtypes = [p, p, p, p, i64, i64, i64, p, p, i64, p, p]
+        L.bro_ref_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, p]
+        L.bro_ref_group_mse.argtypes = [p, p, p, i64, i64, p]
+        for name in ("rotate", "quantize", "decode", "rotate_quantize_mxfp4", "pack_weights",
+                     "gemm_mxfp4", "gemm_mxfp4_points", "linear", "group_mse"):
+            getattr(L, "bro_ref_" + name).restype = ci
+        _lib = L
+    return _lib
+
+
+def _ptr(a: np.ndarray) -> ctypes.c_void_p:
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise ValueError(f"bro_ref_{what} failed with code {rc}")
+
+
+def _as_bf16_bits(x) -> np.ndarray:
+    a = np.ascontiguousarray(x)
+    if a.dtype != np.uint16:
+        raise TypeError("bf16 tensors are passed to the oracle as uint16 bit patterns")
+    if a.ndim != 2:
+        raise ValueError("expected a 2-D array")
+    return a
+
+
+def num_threads() -> int:
+    return int(lib().bro_ref_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    lib().bro_ref_set_num_threads(int(n))
+
+
+def hadamard_norm(block: int) -> np.float32:
+    return np.float32(lib().bro_ref_hadamard_norm(int(block)))
+
+
+def rotate(x_bits, block: int) -> np.ndarray:
+    x = _as_bf16_bits(x_bits)
+    M, K = x.shape
+    y = np.empty((M, K), dtype=np.float32)
+    _check(lib().bro_ref_rotate(_ptr(x), M, K, K, int(block), _ptr(y)), "rotate")
+    return y
+
+
+def quantize(y) -> tuple[np.ndarray, np.ndarray]:
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    rows, K = y.shape
+    codes = np.empty((rows, K // 2), dtype=np.uint8)
+    scales = np.empty((rows, K // MX_GROUP), dtype=np.uint8)
+    _check(lib().bro_ref_quantize(_ptr(y), rows, K, _ptr(codes), _ptr(scales)), "quantize")
+    return codes, scales
+
+
+def decode(codes, scales) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, K), dtype=np.float64)
+    _check(lib().bro_ref_decode(_ptr(codes), _ptr(scales), rows, K, _ptr(out)), "decode")
+    return out
+
+
+def rotate_quantize_mxfp4(x_bits, block: int) -> tuple[np.ndarray, np.ndarray]:
+    x = _as_bf16_bits(x_bits)
+    M, K = x.shape
+    codes = np.empty((M, K // 2), dtype=np.uint8)
+    scales = np.empty((M, K // MX_GROUP), dtype=np.uint8)
+    _check(lib().bro_ref_rotate_quantize_mxfp4(_ptr(x), M, K, K, int(block), _ptr(codes),
+                                               _ptr(scales)), "rotate_quantize_mxfp4")
+    return codes, scales
+
+
+def pack_weights(w_bits, block: int) -> tuple[np.ndarray, np.ndarray]:
+    w = _as_bf16_bits(w_bits)
+    N, K = w.shape
+    codes = np.empty((N, K // 2), dtype=np.uint8)
+    scales = np.empty((N, K // MX_GROUP), dtype=np.uint8)
+    _check(lib().bro_ref_pack_weights(_ptr(w), N, K, K, int(block), _ptr(codes), _ptr(scales)),
+           "pack_weights")
+    return codes, scales
+
+
+def gemm_mxfp4(acodes, ascales, wcodes, wscales) -> tuple[np.ndarray, np.ndarray]:
+    acodes = np.ascontiguousarray(acodes, dtype=np.uint8)
+    ascales = np.ascontiguousarray(ascales, dtype=np.uint8)
+    wcodes = np.ascontiguousarray(wcodes, dtype=np.uint8)
+    wscales = np.ascontiguousarray(wscales, dtype=np.uint8)
+    M, K = acodes.shape[0], acodes.shape[1] * 2
+    N = wcodes.shape[0]
+    y = np.empty((M, N), dtype=np.float64)
+    S = np.empty((M, N), dtype=np.float64)
+    _check(lib().bro_ref_gemm_mxfp4(_ptr(acodes), _ptr(ascales), _ptr(wcodes), _ptr(wscales),
+                                    M, N, K, _ptr(y), _ptr(S)), "gemm_mxfp4")
+    return y, S
+
+
+def gemm_mxfp4_points(acodes, ascales, wcodes, wscales, pm, pn) -> tuple[np.ndarray, np.ndarray]:
+    acodes = np.ascontiguousarray(acodes, dtype=np.uint8)
+    ascales = np.ascontiguousarray(ascales, dtype=np.uint8)
+    wcodes = np.ascontiguousarray(wcodes, dtype=np.uint8)
+    wscales = np.ascontiguousarray(wscales, dtype=np.uint8)
+    pm = np.ascontiguousarray(pm, dtype=np.int64)
+    pn = np.ascontiguousarray(pn, dtype=np.int64)
+    M, K = acodes.shape[0], acodes.shape[1] * 2
+    N = wcodes.shape[0]
+    y = np.empty(pm.shape[0], dtype=np.float64)
+    S = np.empty(pm.shape[0], dtype=np.float64)
+    _check(lib().bro_ref_gemm_mxfp4_points(_ptr(acodes), _ptr(ascales), _ptr(wcodes),
+                                           _ptr(wscales), M, N, K, _ptr(pm), _ptr(pn),
+                                           pm.shape[0], _ptr(y), _ptr(S)), "gemm_mxfp4_points")
+    return y, S
+
+
+def linear(x_bits, block: int, wcodes, wscales) -> tuple[np.ndarray, np.ndarray]:
+    x = _as_bf16_bits(x_bits)
+    wcodes = np.ascontiguousarray(wcodes, dtype=np.uint8)
+    wscales = np.ascontiguousarray(wscales, dtype=np.uint8)
+    M, K = x.shape
+    N = wcodes.shape[0]
+    y = np.empty((M, N), dtype=np.float64)
+    S = np.empty((M, N), dtype=np.float64)
+    _check(lib().bro_ref_linear(_ptr(x), M, K, K, int(block), _ptr(wcodes), _ptr(wscales), N,
+                                _ptr(y), _ptr(S)), "linear")
+    return y, S
+
+
+def group_mse(y, codes, scales) -> np.ndarray:
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    rows, K = y.shape
+    mse = np.empty((rows, K // MX_GROUP), dtype=np.float64)
+    _check(lib().bro_ref_group_mse(_ptr(y), _ptr(codes), _ptr(scales), rows, K, _ptr(mse)),
+           "group_mse")
+    return mse

@@ -1,0 +1,292 @@
+/*
+ * bro_ref.c — CPU oracle (test infrastructure only; see bro_ref.h).
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
+ * -ffp-contract=off matters: every fp32 add/sub/mul below must be one IEEE round-to-nearest
+ * operation, never fused.
+ */
+#include "bro_ref.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define MX_GROUP 32 /* Sec. 4.1: fixed group size of 32 */
+
+/* E2M1 magnitudes for mag = 0..7: exponent field e = mag>>1 (bias 1), mantissa bit m = mag&1.
+ * e == 0 is the subnormal binade (value m * 0.5); otherwise (1 + m/2) * 2^(e-1).  (Sec. 4.1) */
+static const double E2M1_GRID[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+int bro_ref_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void bro_ref_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+static inline float bf16_to_f32(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+static inline uint32_t f32_bits(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  return u;
+}
+
+static int is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+float bro_ref_hadamard_norm(int64_t block) {
+  /* 1/sqrt(B) for B = 2^p is 2^(-p/2): a power of two when p is even, sqrt(2) * 2^(-(p+1)/2)
+   * when p is odd.  Rounding sqrt(2) to fp32 and scaling by a power of two is exact, so this
+   * is the fp32 value nearest to 1/sqrt(B). */
+  int p = 0;
+  while (((int64_t)1 << p) < block) ++p;
+  if ((p & 1) == 0) return ldexpf(1.0f, -p / 2);
+  return ldexpf((float)sqrt(2.0), -(p + 1) / 2);
+}
+
+/* One block: v <- H_B v (Sylvester / natural order) by the fast transform, ascending stride.
+ * Every a+b and a-b is a single fp32 round-to-nearest operation. */
+static void fwht_block(float* v, int64_t B) {
+  for (int64_t h = 1; h < B; h <<= 1) {
+    for (int64_t i = 0; i < B; ++i) {
+      if ((i & h) == 0) {
+        float a = v[i];
+        float b = v[i + h];
+        v[i] = a + b;
+        v[i + h] = a - b;
+      }
+    }
+  }
+}
+
+int bro_ref_rotate(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int block, float* y) {
+  if (!x || !y) return 1;
+  if (M < 0 || K <= 0 || ldx < K) return 2;
+  int64_t B = block == 0 ? K : block;
+  if (!is_pow2(B) || K % B != 0) return 2;
+  const float c = bro_ref_hadamard_norm(B);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m) {
+    float* row = y + m * K;
+    for (int64_t k = 0; k < K; ++k) row[k] = bf16_to_f32(x[m * ldx + k]);
+    for (int64_t b0 = 0; b0 < K; b0 += B) {
+      fwht_block(row + b0, B);
+      for (int64_t i = 0; i < B; ++i) row[b0 + i] = row[b0 + i] * c; /* one multiply, at the end */
+    }
+  }
+  return 0;
+}
+
+/* Round a non-negative scaled magnitude r onto the E2M1 grid, nearest, ties to the even code,
+ * saturating at 6 (mag 7). */
+static inline unsigned e2m1_round(float r) {
+  if (r <= 0.25f) return 0; /* tie .25 -> 0   (even) */
+  if (r < 0.75f) return 1;
+  if (r <= 1.25f) return 2; /* ties .75, 1.25 -> 1.0 (even) */
+  if (r < 1.75f) return 3;
+  if (r <= 2.5f) return 4; /* ties 1.75, 2.5 -> 2.0 (even) */
+  if (r < 3.5f) return 5;
+  if (r <= 5.0f) return 6; /* ties 3.5, 5 -> 4.0 (even) */
+  return 7;                /* (5, inf): 6.0, saturating */
+}
+
+static void quantize_group(const float* y, uint8_t* codes16, uint8_t* scale) {
+  float amax = 0.0f;
+  for (int i = 0; i < MX_GROUP; ++i) {
+    float a = fabsf(y[i]);
+    if (a > amax) amax = a;
+  }
+  /* floor(log2(amax)) for a normal fp32 is its biased exponent field minus 127.  The shared
+   * exponent is that minus emax_elem (= 2 for E2M1), clamped below at the smallest E8M0 value. */
+  int ef = (int)((f32_bits(amax) >> 23) & 0xFF);
+  int s = ef - 2;
+  if (s < 0) s = 0;
+  int E = s - 127;
+  *scale = (uint8_t)s;
+  for (int i = 0; i < MX_GROUP; i += 2) {
+    unsigned c[2];
+    for (int j = 0; j < 2; ++j) {
+      float v = y[i + j];
+      float r = ldexpf(fabsf(v), -E); /* exact power-of-two scaling */
+      unsigned mag = e2m1_round(r);
+      unsigned sign = (f32_bits(v) >> 31) & 1u;
+      c[j] = (sign << 3) | mag;
+    }
+    codes16[i / 2] = (uint8_t)(c[0] | (c[1] << 4));
+  }
+}
+
+int bro_ref_quantize(const float* y, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales) {
+  if (!y || !codes || !scales) return 1;
+  if (rows < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  const int64_t ng = K / MX_GROUP;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t g = 0; g < ng; ++g)
+      quantize_group(y + r * K + g * MX_GROUP, codes + r * (K / 2) + g * (MX_GROUP / 2),
+                     scales + r * ng + g);
+  return 0;
+}
+
+static inline double decode_one(unsigned code, int E) {
+  double v = ldexp(E2M1_GRID[code & 7u], E);
+  return (code & 8u) ? -v : v;
+}
+
+int bro_ref_decode(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K,
+                   double* out) {
+  if (!codes || !scales || !out) return 1;
+  if (rows < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  const int64_t ng = K / MX_GROUP;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t k = 0; k < K; ++k) {
+      uint8_t byte = codes[r * (K / 2) + k / 2];
+      unsigned code = (k & 1) ? (byte >> 4) : (byte & 0xF);
+      int E = (int)scales[r * ng + k / MX_GROUP] - 127;
+      out[r * K + k] = decode_one(code, E);
+    }
+  return 0;
+}
+
+int bro_ref_rotate_quantize_mxfp4(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
+                                  int block, uint8_t* codes, uint8_t* scales) {
+  if (!x || !codes || !scales) return 1;
+  if (M < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  if (M == 0) return 0;
+  float* y = (float*)malloc((size_t)M * (size_t)K * sizeof(float));
+  if (!y) return 3;
+  int rc = bro_ref_rotate(x, M, K, ldx, block, y);
+  if (rc == 0) rc = bro_ref_quantize(y, M, K, codes, scales);
+  free(y);
+  return rc;
+}
+
+int bro_ref_pack_weights(const uint16_t* w, int64_t N, int64_t K, int64_t ldw, int block,
+                         uint8_t* wcodes, uint8_t* wscales) {
+  /* "Weights are rotated and quantised the same way": rows of W are output channels, the
+   * rotation acts on the K axis exactly as for activations (R_block R_block^T = I, Eq. 1). */
+  return bro_ref_rotate_quantize_mxfp4(w, N, K, ldw, block, wcodes, wscales);
+}
+
+int bro_ref_gemm_mxfp4(const uint8_t* acodes, const uint8_t* ascales, const uint8_t* wcodes,
+                       const uint8_t* wscales, int64_t M, int64_t N, int64_t K, double* y,
+                       double* S) {
+  if (!acodes || !ascales || !wcodes || !wscales || !y) return 1;
+  if (M < 0 || N < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  if (M == 0 || N == 0) return 0;
+  double* A = (double*)malloc((size_t)M * (size_t)K * sizeof(double));
+  double* W = (double*)malloc((size_t)N * (size_t)K * sizeof(double));
+  if (!A || !W) {
+    free(A);
+    free(W);
+    return 3;
+  }
+  bro_ref_decode(acodes, ascales, M, K, A);
+  bro_ref_decode(wcodes, wscales, N, K, W);
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t n = 0; n < N; ++n) {
+      double acc = 0.0, sabs = 0.0;
+      for (int64_t k = 0; k < K; ++k) {
+        double p = A[m * K + k] * W[n * K + k]; /* exact in fp64 */
+        acc += p;
+        sabs += fabs(p);
+      }
+      y[m * N + n] = acc;
+      if (S) S[m * N + n] = sabs;
+    }
+  free(A);
+  free(W);
+  return 0;
+}
+
+int bro_ref_gemm_mxfp4_points(const uint8_t* acodes, const uint8_t* ascales,
+                              const uint8_t* wcodes, const uint8_t* wscales, int64_t M,
+                              int64_t N, int64_t K, const int64_t* pm, const int64_t* pn,
+                              int64_t npoints, double* y, double* S) {
+  if (!acodes || !ascales || !wcodes || !wscales || !pm || !pn || !y) return 1;
+  if (M <= 0 || N <= 0 || K <= 0 || K % MX_GROUP != 0 || npoints < 0) return 2;
+  const int64_t ng = K / MX_GROUP;
+  for (int64_t p = 0; p < npoints; ++p)
+    if (pm[p] < 0 || pm[p] >= M || pn[p] < 0 || pn[p] >= N) return 2;
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < npoints; ++p) {
+    const int64_t m = pm[p], n = pn[p];
+    double acc = 0.0, sabs = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+      uint8_t ab = acodes[m * (K / 2) + k / 2];
+      uint8_t wb = wcodes[n * (K / 2) + k / 2];
+      unsigned ac = (k & 1) ? (ab >> 4) : (ab & 0xF);
+      unsigned wc = (k & 1) ? (wb >> 4) : (wb & 0xF);
+      double a = decode_one(ac, (int)ascales[m * ng + k / MX_GROUP] - 127);
+      double w = decode_one(wc, (int)wscales[n * ng + k / MX_GROUP] - 127);
+      double prod = a * w;
+      acc += prod;
+      sabs += fabs(prod);
+    }
+    y[p] = acc;
+    if (S) S[p] = sabs;
+  }
+  return 0;
+}
+
+int bro_ref_linear(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int block,
+                   const uint8_t* wcodes, const uint8_t* wscales, int64_t N, double* y,
+                   double* S) {
+  if (!x || !wcodes || !wscales || !y) return 1;
+  if (M < 0 || N < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  if (M == 0 || N == 0) return 0;
+  uint8_t* ac = (uint8_t*)malloc((size_t)M * (size_t)(K / 2));
+  uint8_t* as = (uint8_t*)malloc((size_t)M * (size_t)(K / MX_GROUP));
+  if (!ac || !as) {
+    free(ac);
+    free(as);
+    return 3;
+  }
+  int rc = bro_ref_rotate_quantize_mxfp4(x, M, K, ldx, block, ac, as);
+  if (rc == 0) rc = bro_ref_gemm_mxfp4(ac, as, wcodes, wscales, M, N, K, y, S);
+  free(ac);
+  free(as);
+  return rc;
+}
+
+int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scales,
+                      int64_t rows, int64_t K, double* mse) {
+  if (!y || !codes || !scales || !mse) return 1;
+  if (rows < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
+  const int64_t ng = K / MX_GROUP;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t g = 0; g < ng; ++g) {
+      int E = (int)scales[r * ng + g] - 127;
+      double acc = 0.0;
+      for (int i = 0; i < MX_GROUP; ++i) {
+        int64_t k = g * MX_GROUP + i;
+        uint8_t byte = codes[r * (K / 2) + k / 2];
+        unsigned code = (k & 1) ? (byte >> 4) : (byte & 0xF);
+        double d = (double)y[r * K + k] - decode_one(code, E);
+        acc += d * d;
+      }
+      mse[r * ng + g] = acc / MX_GROUP;
+    }
+  return 0;
+}

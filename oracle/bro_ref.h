@@ -1,0 +1,98 @@
+/*
+ * bro_ref — CPU oracle for the block-rotated MXFP4 W4A4 linear layer.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, obviously-correct restatement of what the
+ * method computes, written from the paper's text.  It shares no code, header, table or helper
+ * with the CUDA library; only the tests, the smoke check and the benchmark's CPU-baseline leg
+ * may call it.  The product path never routes through it.
+ *
+ * What it follows:
+ *   - Block-diagonal orthogonal rotation R_block = diag(R_1..R_B), R_i^T R_i = I, block aligned
+ *     with the MX group                                         (paper Sec. 4.3, Eq. 1)
+ *   - R_i is a Hadamard matrix (Sylvester construction, normalised by 1/sqrt(block)); the
+ *     online transform is a fast Hadamard transform             (Sec. 4.3 "Reduced online
+ *     computing", Sec. 5.1, Sec. 6)
+ *   - MXFP4: E2M1 elements (1 sign, 2 exponent, 1 mantissa bit), groups of 32 that share one
+ *     E8M0 power-of-two scale, symmetric                        (Sec. 4.1)
+ *   - Scale and rounding rule: the OCP Microscaling rule the paper cites in Sec. 1:
+ *     shared exponent = floor(log2(amax)) - emax_elem with emax_elem = 2 for E2M1, elements
+ *     rounded to nearest, ties to even, saturating at +-6.
+ *   - W4A4 linear: y = Q(x R) . Q(W R)^T                          (Sec. 1, Sec. 4.2, Sec. 4.3)
+ *
+ * Pin status: every function below is pinned by the CPU tests (orthogonality, norm
+ * preservation, exact inversion, closed forms, an independent O(B^2) definition, worked E2M1
+ * examples, brute-force nearest-grid search, idempotence, integer-matmul special cases,
+ * the per-element error bound).  One exception: bro_ref_group_mse's *qualitative ordering*
+ * between rotation sizes (Sec. 5.2, Fig. 6/7) is "parity unpinned" — the paper prints figures,
+ * not numbers; the MSE arithmetic itself is pinned against a numpy restatement.
+ *
+ * Data formats (all host pointers):
+ *   bf16 input        : uint16_t, the upper 16 bits of the IEEE fp32 pattern.
+ *   codes             : uint8_t [rows, K/2]; byte j of a row holds element 2j in bits 0..3 and
+ *                       element 2j+1 in bits 4..7; a code is sign<<3 | mag, mag 0..7 <->
+ *                       {0, .5, 1, 1.5, 2, 3, 4, 6}.
+ *   scales            : uint8_t [rows, K/32], row-major; byte = E + 127, value 2^E.
+ * All functions return 0 on success, non-zero on a bad argument.
+ */
+#ifndef BRO_REF_H
+#define BRO_REF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Number of OpenMP threads the oracle will use (1 if built without OpenMP). */
+int bro_ref_num_threads(void);
+void bro_ref_set_num_threads(int n);
+
+/* The fp32 constant c_B = nearest fp32 to 1/sqrt(block) used to normalise H_B. */
+float bro_ref_hadamard_norm(int64_t block);
+
+/* Rotation only (Eq. 1 with Hadamard R_i): y[m, :] = x[m, :] R_block, fp32 out [M, K] dense.
+ * block in {2^k}; block == 0 means block = K (global rotation, K must be a power of two). */
+int bro_ref_rotate(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                   float* y);
+
+/* MXFP4 quantisation of fp32 rows (Sec. 4.1): per group of 32, E8M0 scale + 32 E2M1 codes. */
+int bro_ref_quantize(const float* y, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales);
+
+/* Decode codes+scales to fp64 values [rows, K] (exact). */
+int bro_ref_decode(const uint8_t* codes, const uint8_t* scales, int64_t rows, int64_t K,
+                   double* out);
+
+/* Activation path: rotate then quantise. */
+int bro_ref_rotate_quantize_mxfp4(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                                  int block, uint8_t* codes, uint8_t* scales);
+
+/* Weight path: identical arithmetic applied to the rows of W[N, K] (offline). */
+int bro_ref_pack_weights(const uint16_t* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                         uint8_t* wcodes, uint8_t* wscales);
+
+/* y[m,n] = sum_k deq_a[m,k] * deq_w[n,k] in fp64, index order; S[m,n] = sum_k |deq_a*deq_w|.
+ * S may be NULL. */
+int bro_ref_gemm_mxfp4(const uint8_t* acodes, const uint8_t* ascales, const uint8_t* wcodes,
+                       const uint8_t* wscales, int64_t M, int64_t N, int64_t K, double* y,
+                       double* S);
+
+/* The same sums for a list of (m, n) points only — for sampled parity at large sizes. */
+int bro_ref_gemm_mxfp4_points(const uint8_t* acodes, const uint8_t* ascales,
+                              const uint8_t* wcodes, const uint8_t* wscales, int64_t M,
+                              int64_t N, int64_t K, const int64_t* pm, const int64_t* pn,
+                              int64_t npoints, double* y, double* S);
+
+/* Whole layer: rotate+quantise x, then the GEMM against packed weights. */
+int bro_ref_linear(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                   const uint8_t* wcodes, const uint8_t* wscales, int64_t N, double* y,
+                   double* S);
+
+/* Per-group quantisation error: mse[r, g] = mean_{i in group} (y[r,i] - deq[r,i])^2, fp64. */
+int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scales,
+                      int64_t rows, int64_t K, double* mse);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BRO_REF_H */
