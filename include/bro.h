@@ -1,0 +1,152 @@
+/*
+ * bro.h — C ABI of libbro: the W4A4 MXFP4 linear layer with block-Hadamard rotation on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The operations follow "Block Rotation is All You Need for MXFP4 Quantization"
+ * (arXiv 2511.04214):
+ *   - rotation   x -> x R_block, R_block = diag(R_1..R_B) with orthogonal blocks aligned with
+ *                the MX group (Sec. 4.3, Eq. 1); R_i = H_block / sqrt(block), H the Sylvester
+ *                Hadamard matrix, applied as a fast transform (Sec. 4.3 "Reduced online
+ *                computing", Sec. 5.1);
+ *   - MXFP4      E2M1 elements, groups of 32 sharing one E8M0 power-of-two scale (Sec. 4.1),
+ *                scale exponent = floor(log2 amax) - 2, round-to-nearest-even, saturate at +-6
+ *                (the OCP Microscaling rule the paper cites in Sec. 1);
+ *   - W4A4       y = Q(x R) Q(W R)^T with fp32 accumulation (Sec. 1, Sec. 4.2).
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
+ *     The library allocates no device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     enqueue work and return without synchronising.  The returned status covers argument
+ *     validation and launch errors only.
+ *   - Every device-side wait is bounded.  If one expires (which indicates a bug or a broken
+ *     device, never a data condition) the kernel records BRO_ERR_TIMEOUT in a device-side
+ *     status word and returns; bro_last_device_status() reads and clears that word.
+ *   - No exception crosses this boundary.  Invalid arguments return an error code; they never
+ *     lead to undefined behaviour.  M == 0 or N == 0 returns BRO_OK without a launch.
+ *   - bf16 tensors are row-major with a leading dimension in ELEMENTS.
+ *
+ * Data formats
+ *   codes   uint8 [rows, K/2], row-major, dense.  Byte j of a row holds element 2j in bits 0..3
+ *           and element 2j+1 in bits 4..7.  A code is sign<<3 | mag, mag 0..7 <->
+ *           {0, 0.5, 1, 1.5, 2, 3, 4, 6}.  The sign bit of a value that rounds to zero is kept.
+ *   scales  uint8, one per (row, group of 32): byte = E + 127 for the scale 2^E.  0xFF is never
+ *           produced for finite input.
+ *           BRO_LAYOUT_CANONICAL: [rows, K/32] row-major.
+ *           BRO_LAYOUT_GEMM: the order the tensor core reads.  Rows are padded to a multiple of
+ *           128 and K to a multiple of 256; the buffer is an array [ceil(rows/128)][KB] of
+ *           512-byte blocks, KB = 2*ceil(K/256), block (i, j) covering rows 128i..128i+127 and
+ *           groups 4j..4j+3; inside a block the byte for (row r, group g) sits at
+ *           (r%32)*16 + ((r%128)/32)*4 + (g%4).  Padding bytes are written as 0.
+ *           bro_scale_offset() returns the byte offset of one (row, group) in either layout.
+ */
+#ifndef BRO_H
+#define BRO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BRO_OK = 0,
+  BRO_ERR_NULL = 1,        /* a required pointer is NULL */
+  BRO_ERR_SHAPE = 2,       /* a size, leading dimension or block value is not allowed */
+  BRO_ERR_ALIGN = 3,       /* a pointer or leading dimension is not aligned as required */
+  BRO_ERR_UNSUPPORTED = 4, /* valid request that this build does not implement */
+  BRO_ERR_WORKSPACE = 5,   /* workspace too small */
+  BRO_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed */
+  BRO_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired */
+  BRO_ERR_ARCH = 8         /* the current device is not compute capability 10.x */
+} bro_status;
+
+typedef enum { BRO_LAYOUT_CANONICAL = 0, BRO_LAYOUT_GEMM = 1 } bro_layout;
+typedef enum { BRO_OUT_BF16 = 0, BRO_OUT_F32 = 1 } bro_out_dtype;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* bro_status_string(bro_status s);
+
+/* rows*K/2: bytes of a packed code tensor. */
+size_t bro_codes_bytes(int64_t rows, int64_t K);
+/* Bytes of a scale tensor in the given layout (padded for BRO_LAYOUT_GEMM). 0 on bad input. */
+size_t bro_scales_bytes(int64_t rows, int64_t K, bro_layout layout);
+/* Byte offset of the scale of (row, group) inside a scale tensor of `rows` x K. */
+size_t bro_scale_offset(int64_t row, int64_t group, int64_t rows, int64_t K, bro_layout layout);
+/* Workspace bro_gemm_mxfp4 needs for this problem (may be 0). */
+size_t bro_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+/* Workspace bro_linear needs: quantised activations (codes + GEMM-layout scales) + the GEMM's. */
+size_t bro_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/* Synchronises `stream`, then returns and clears the device-side status word of the current
+ * device: BRO_OK, or BRO_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call.
+ * BRO_ERR_CUDA if the synchronisation itself reports an error. */
+bro_status bro_last_device_status(void* stream);
+
+/*
+ * Online activation path (Sec. 4.3 Eq. 1 + Sec. 4.1): for every row of x[M, K] (bf16) and every
+ * aligned block of `block` channels, y = (H_block x) / sqrt(block) in fp32 — butterflies in
+ * ascending stride order, one multiply by the fp32 nearest 1/sqrt(block) at the end — then each
+ * group of 32 values of y is quantised to MXFP4.
+ *   block   32, 64 or 128; or 0 for block = K (global rotation; K must then be a power of two,
+ *           32 <= K <= 32768).
+ *   ldx     row stride of x in elements, >= K, multiple of 8.
+ *   codes   out, [M, K/2] bytes, 16-byte aligned.
+ *   scales  out, bro_scales_bytes(M, K, layout) bytes, 16-byte aligned.
+ * Requirements: K % 32 == 0, K % block == 0, x 16-byte aligned.
+ */
+bro_status bro_rotate_quantize_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                                     int block, void* codes, void* scales, bro_layout layout,
+                                     void* stream);
+
+/*
+ * Offline weight path: the same arithmetic applied to the rows of w[N, K] (the rotation acts on
+ * the K axis of both operands, so (x R)(W R)^T = x W^T before quantisation, Eq. 1).  Scales are
+ * written in BRO_LAYOUT_GEMM.
+ */
+bro_status bro_pack_weights(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                            void* wcodes, void* wscales, void* stream);
+
+/*
+ * Block-scaled MXFP4 x MXFP4 GEMM (Sec. 1 W4A4; Sec. 4.2):
+ *   y[m, n] = sum_g 2^(Ea[m,g] + Ew[n,g]) * sum_{k in group g} a[m,k] * w[n,k]
+ * with fp32 accumulation on the tensor cores and the result written as bf16 (round to nearest
+ * even) or fp32.
+ *   acodes/wcodes    [M, K/2] and [N, K/2] bytes, 128-byte aligned.
+ *   ascales/wscales  BRO_LAYOUT_GEMM, 128-byte aligned.
+ *   y                [M, ldy] of out_dtype, 16-byte aligned; ldy >= N, ldy*sizeof(elem) % 16 == 0.
+ *   workspace        bro_gemm_workspace_bytes(M, N, K) bytes (may be NULL when that is 0).
+ * Requirements: K % 32 == 0.
+ */
+bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* wcodes,
+                          const void* wscales, int64_t M, int64_t N, int64_t K, void* y,
+                          int64_t ldy, bro_out_dtype out_dtype, void* workspace,
+                          size_t workspace_bytes, void* stream);
+
+/*
+ * The whole layer on one stream: bro_rotate_quantize_mxfp4(x) into the workspace, then
+ * bro_gemm_mxfp4 against weights packed by bro_pack_weights with the same `block`.
+ *   workspace   bro_linear_workspace_bytes(M, N, K) bytes, 1024-byte aligned.
+ *   y_bf16      [M, ldy] bf16.
+ */
+bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                      const void* wcodes, const void* wscales, int64_t N, void* y_bf16,
+                      int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * bro_linear for a caller whose activations and result live in HOST memory (pinned memory gives
+ * asynchronous copies).  Copies x_host[M, K] (dense, ldx = K) to the device staging buffer,
+ * runs bro_linear, and copies y[M, N] (dense) back to y_host, all on `stream`.
+ *   x_stage  device, M*K*2 bytes;  y_stage  device, M*N*2 bytes;  both 16-byte aligned.
+ * The call returns after enqueuing; synchronise the stream before reading y_host.
+ */
+bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block,
+                           const void* wcodes, const void* wscales, int64_t N,
+                           void* y_host_bf16, void* x_stage, void* y_stage, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BRO_H */

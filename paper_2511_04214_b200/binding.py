@@ -1,0 +1,178 @@
+"""ctypes binding for libbro — argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory owned by the caller), passes raw pointers
+and sizes to the C ABI declared in ``include/bro.h`` and raises :class:`BroError` on a non-zero
+status.  No step of the method runs in Python or in PyTorch ops, and there is no CPU fallback:
+if the shared library is missing the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libbro.so")
+
+LAYOUT_CANONICAL = 0
+LAYOUT_GEMM = 1
+OUT_BF16 = 0
+OUT_F32 = 1
+
+EXPORTS = [
+    "bro_status_string", "bro_codes_bytes", "bro_scales_bytes", "bro_scale_offset",
+    "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
+    "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
+    "bro_linear_host",
+]
+
+
+class BroError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_SO):
+        raise ImportError(
+            f"{_SO} is missing: build it with `python -m paper_2511_04214_b200.build` "
+            "(there is no fallback path)")
+    L = ctypes.CDLL(_SO)
+    i64, p, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.bro_status_string.restype = ctypes.c_char_p
+    L.bro_status_string.argtypes = [ci]
+    L.bro_codes_bytes.restype = sz
+    L.bro_codes_bytes.argtypes = [i64, i64]
+    L.bro_scales_bytes.restype = sz
+    L.bro_scales_bytes.argtypes = [i64, i64, ci]
+    L.bro_scale_offset.restype = sz
+    L.bro_scale_offset.argtypes = [i64, i64, i64, i64, ci]
+    L.bro_gemm_workspace_bytes.restype = sz
+    L.bro_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+    L.bro_linear_workspace_bytes.restype = sz
+    L.bro_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.bro_last_device_status.restype = ci
+    L.bro_last_device_status.argtypes = [p]
+    L.bro_rotate_quantize_mxfp4.restype = ci
+    L.bro_rotate_quantize_mxfp4.argtypes = [p, i64, i64, i64, ci, p, p, ci, p]
+    L.bro_pack_weights.restype = ci
+    L.bro_pack_weights.argtypes = [p, i64, i64, i64, ci, p, p, p]
+    L.bro_gemm_mxfp4.restype = ci
+    L.bro_gemm_mxfp4.argtypes = [p, p, p, p, i64, i64, i64, p, i64, ci, p, sz, p]
+    L.bro_linear.restype = ci
+    L.bro_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p, sz, p]
+    L.bro_linear_host.restype = ci
+    L.bro_linear_host.argtypes = [p, i64, i64, ci, p, p, i64, p, p, p, p, sz, p]
+    return L
+
+
+lib = _load()
+
+
+def status_string(code: int) -> str:
+    return lib.bro_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise BroError(code, where)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t) -> ctypes.c_void_p:
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def codes_bytes(rows: int, K: int) -> int:
+    return int(lib.bro_codes_bytes(rows, K))
+
+
+def scales_bytes(rows: int, K: int, layout: int) -> int:
+    return int(lib.bro_scales_bytes(rows, K, layout))
+
+
+def scale_offset(row: int, group: int, rows: int, K: int, layout: int) -> int:
+    return int(lib.bro_scale_offset(row, group, rows, K, layout))
+
+
+def gemm_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib.bro_gemm_workspace_bytes(M, N, K))
+
+
+def linear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib.bro_linear_workspace_bytes(M, N, K))
+
+
+def last_device_status(stream=None) -> int:
+    return int(lib.bro_last_device_status(_stream(stream)))
+
+
+def alloc_codes(rows: int, K: int, device="cuda") -> torch.Tensor:
+    return torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
+
+
+def alloc_scales(rows: int, K: int, layout: int, device="cuda") -> torch.Tensor:
+    return torch.empty(scales_bytes(rows, K, layout), dtype=torch.uint8, device=device)
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """uint8 buffer of at least ``nbytes`` whose start is 1024-byte aligned."""
+    raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-raw.data_ptr()) % 1024
+    return raw[off:off + max(nbytes, 1)]
+
+
+def rotate_quantize_mxfp4(x: torch.Tensor, block: int, codes: torch.Tensor, scales: torch.Tensor,
+                          layout: int = LAYOUT_GEMM, stream=None) -> None:
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    _check(lib.bro_rotate_quantize_mxfp4(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K),
+                                         block, _ptr(codes), _ptr(scales), layout, _stream(stream)),
+           "bro_rotate_quantize_mxfp4")
+
+
+def pack_weights(w: torch.Tensor, block: int, wcodes: torch.Tensor, wscales: torch.Tensor,
+                 stream=None) -> None:
+    assert w.dtype == torch.bfloat16 and w.dim() == 2 and w.stride(1) == 1
+    N, K = w.shape
+    _check(lib.bro_pack_weights(_ptr(w), N, K, w.stride(0) if N > 1 else max(w.stride(0), K), block,
+                                _ptr(wcodes), _ptr(wscales), _stream(stream)), "bro_pack_weights")
+
+
+def gemm_mxfp4(acodes, ascales, wcodes, wscales, M: int, N: int, K: int, y: torch.Tensor,
+               workspace=None, stream=None) -> None:
+    out = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
+    assert y.dtype in (torch.bfloat16, torch.float32) and y.stride(1) == 1
+    wsb = 0 if workspace is None else workspace.numel()
+    _check(lib.bro_gemm_mxfp4(_ptr(acodes), _ptr(ascales), _ptr(wcodes), _ptr(wscales), M, N, K,
+                              _ptr(y), y.stride(0) if M > 1 else max(y.stride(0), N), out,
+                              _ptr(workspace), wsb, _stream(stream)), "bro_gemm_mxfp4")
+
+
+def linear(x: torch.Tensor, block: int, wcodes, wscales, N: int, y: torch.Tensor,
+           workspace: torch.Tensor, stream=None) -> None:
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+    M, K = x.shape
+    _check(lib.bro_linear(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K), block,
+                          _ptr(wcodes), _ptr(wscales), N, _ptr(y),
+                          y.stride(0) if M > 1 else max(y.stride(0), N), _ptr(workspace),
+                          workspace.numel(), _stream(stream)), "bro_linear")
+
+
+def linear_host(x_host: torch.Tensor, block: int, wcodes, wscales, N: int, y_host: torch.Tensor,
+                x_stage: torch.Tensor, y_stage: torch.Tensor, workspace: torch.Tensor,
+                stream=None) -> None:
+    """Host-buffer variant: x_host / y_host are (ideally pinned) CPU bf16 tensors."""
+    assert x_host.device.type == "cpu" and y_host.device.type == "cpu"
+    assert x_host.is_contiguous() and y_host.is_contiguous()
+    M, K = x_host.shape
+    _check(lib.bro_linear_host(_ptr(x_host), M, K, block, _ptr(wcodes), _ptr(wscales), N,
+                               _ptr(y_host), _ptr(x_stage), _ptr(y_stage), _ptr(workspace),
+                               workspace.numel(), _stream(stream)), "bro_linear_host")

@@ -1,0 +1,283 @@
+// libbro: C ABI over the two sm_100a kernels (see include/bro.h for the contract).
+// Host-side work only: argument validation, TMA tensor-map encoding, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "../../include/bro.h"
+#include "bro_common.cuh"
+#include "rotate_quantize.cuh"
+#include "rotate_quantize_global.cuh"
+#include "gemm_mxfp4.cuh"
+
+namespace {
+
+using bro::rq::Params;
+
+constexpr int64_t kGroup = 32;
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+
+// ---- device / driver plumbing ------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+struct DeviceInfo {
+  bool ok = false;
+  int sm_count = 0;
+};
+
+// Per-device facts, looked up once per device.
+bro_status device_info(DeviceInfo* out) {
+  static DeviceInfo cache[64];
+  static bool known[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return BRO_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return BRO_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!known[dev]) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BRO_ERR_CUDA;
+    cache[dev].ok = (prop.major == 10);
+    cache[dev].sm_count = prop.multiProcessorCount;
+    known[dev] = true;
+  }
+  *out = cache[dev];
+  return out->ok ? BRO_OK : BRO_ERR_ARCH;
+}
+
+// 2-D row-major tensor map: dims {inner, rows}, row pitch in bytes, box {box_inner, box_rows}.
+bro_status make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t elem_bytes, const void* base,
+                       uint64_t inner, uint64_t rows, uint64_t pitch_bytes, uint32_t box_inner,
+                       uint32_t box_rows, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return BRO_ERR_CUDA;
+  cuuint64_t dims[2] = {inner, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  (void)elem_bytes;
+  CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BRO_OK : BRO_ERR_CUDA;
+}
+
+template <typename K>
+bro_status set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
+             ? BRO_OK
+             : BRO_ERR_CUDA;
+}
+
+int64_t gemm_scale_kblocks(int64_t K) { return 2 * ceil_div(K, 256); }
+
+// ---- rotate + quantise ---------------------------------------------------------------------------
+bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, int block,
+                                  void* codes, void* scales, bro_layout layout, cudaStream_t st) {
+  if (!x || !codes || !scales) return BRO_ERR_NULL;
+  if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (layout != BRO_LAYOUT_CANONICAL && layout != BRO_LAYOUT_GEMM) return BRO_ERR_SHAPE;
+  const int64_t B = block == 0 ? K : block;
+  if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  if (K % B != 0) return BRO_ERR_SHAPE;
+  if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
+  if (ldx % 8 != 0 || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16)) return BRO_ERR_ALIGN;
+  if (M == 0) return BRO_OK;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+
+  if (B > 128) {
+    return bro::rqg::launch(x, M, K, ldx, codes, scales, layout, gemm_scale_kblocks(K), di.sm_count, st);
+  }
+
+  CUtensorMap tmx;
+  rc = make_map_2d(&tmx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, (uint64_t)K, (uint64_t)M,
+                   (uint64_t)ldx * 2, bro::rq::kBoxCols, bro::rq::kTileRows, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (rc != BRO_OK) return rc;
+
+  Params p;
+  p.M = M;
+  p.K = K;
+  p.tiles_m = ceil_div(M, bro::rq::kTileRows);
+  p.tiles_k = layout == BRO_LAYOUT_GEMM ? gemm_scale_kblocks(K) : ceil_div(K, bro::rq::kTileCols);
+  p.codes = static_cast<uint8_t*>(codes);
+  p.scales = static_cast<uint8_t*>(scales);
+  p.scale_kblocks = gemm_scale_kblocks(K);
+  p.layout = (int)layout;
+  const int64_t tiles = p.tiles_m * p.tiles_k;
+  const int grid = (int)(tiles < di.sm_count ? tiles : di.sm_count);
+
+  auto go = [&](auto kernel) -> bro_status {
+    static thread_local bool attr_done[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_done[dev]) {
+      bro_status r = set_smem(kernel, bro::rq::kSmemBytes);
+      if (r != BRO_OK) return r;
+      attr_done[dev] = true;
+    }
+    kernel<<<grid, bro::rq::kThreads, bro::rq::kSmemBytes, st>>>(tmx, p);
+    return cudaGetLastError() == cudaSuccess ? BRO_OK : BRO_ERR_CUDA;
+  };
+  switch (B) {
+    case 32: return go(bro::rq::rotate_quantize_kernel<5>);
+    case 64: return go(bro::rq::rotate_quantize_kernel<6>);
+    default: return go(bro::rq::rotate_quantize_kernel<7>);
+  }
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+const char* bro_status_string(bro_status s) {
+  switch (s) {
+    case BRO_OK: return "BRO_OK";
+    case BRO_ERR_NULL: return "BRO_ERR_NULL";
+    case BRO_ERR_SHAPE: return "BRO_ERR_SHAPE";
+    case BRO_ERR_ALIGN: return "BRO_ERR_ALIGN";
+    case BRO_ERR_UNSUPPORTED: return "BRO_ERR_UNSUPPORTED";
+    case BRO_ERR_WORKSPACE: return "BRO_ERR_WORKSPACE";
+    case BRO_ERR_CUDA: return "BRO_ERR_CUDA";
+    case BRO_ERR_TIMEOUT: return "BRO_ERR_TIMEOUT";
+    case BRO_ERR_ARCH: return "BRO_ERR_ARCH";
+  }
+  return "BRO_ERR_UNKNOWN";
+}
+
+size_t bro_codes_bytes(int64_t rows, int64_t K) {
+  if (rows < 0 || K <= 0 || K % kGroup != 0) return 0;
+  return (size_t)rows * (size_t)(K / 2);
+}
+
+size_t bro_scales_bytes(int64_t rows, int64_t K, bro_layout layout) {
+  if (rows < 0 || K <= 0 || K % kGroup != 0) return 0;
+  if (layout == BRO_LAYOUT_CANONICAL) return (size_t)rows * (size_t)(K / kGroup);
+  if (layout == BRO_LAYOUT_GEMM) return (size_t)ceil_div(rows, 128) * (size_t)gemm_scale_kblocks(K) * 512;
+  return 0;
+}
+
+size_t bro_scale_offset(int64_t row, int64_t group, int64_t rows, int64_t K, bro_layout layout) {
+  (void)rows;
+  if (layout == BRO_LAYOUT_CANONICAL) return (size_t)(row * (K / kGroup) + group);
+  return (size_t)(((row / 128) * gemm_scale_kblocks(K) + group / 4) * 512 + (row % 32) * 16 +
+                  ((row % 128) / 32) * 4 + (group % 4));
+}
+
+size_t bro_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  return bro::gemm::workspace_bytes(M, N, K);
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t bro_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return 0;
+  return align_up(bro_codes_bytes(M, K), 1024) + align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 1024) +
+         align_up(bro_gemm_workspace_bytes(M, N, K), 1024);
+}
+
+bro_status bro_last_device_status(void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BRO_ERR_CUDA;
+  unsigned int v = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&v, bro::g_device_status, sizeof(v)) != cudaSuccess) return BRO_ERR_CUDA;
+  if (v != 0 && cudaMemcpyToSymbol(bro::g_device_status, &zero, sizeof(zero)) != cudaSuccess)
+    return BRO_ERR_CUDA;
+  return (bro_status)(v & 0xFF);
+}
+
+bro_status bro_rotate_quantize_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                     void* codes, void* scales, bro_layout layout, void* stream) {
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, codes, scales, layout,
+                                static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_pack_weights(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                            void* wcodes, void* wscales, void* stream) {
+  return launch_rotate_quantize(w_bf16, N, K, ldw, block, wcodes, wscales, BRO_LAYOUT_GEMM,
+                                static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* wcodes,
+                          const void* wscales, int64_t M, int64_t N, int64_t K, void* y, int64_t ldy,
+                          bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+  if (!acodes || !ascales || !wcodes || !wscales || !y) return BRO_ERR_NULL;
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0 || ldy < N) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (out_dtype != BRO_OUT_BF16 && out_dtype != BRO_OUT_F32) return BRO_ERR_SHAPE;
+  const int64_t esz = out_dtype == BRO_OUT_BF16 ? 2 : 4;
+  if (!aligned(acodes, 128) || !aligned(wcodes, 128) || !aligned(ascales, 128) || !aligned(wscales, 128) ||
+      !aligned(y, 16) || (ldy * esz) % 16 != 0)
+    return BRO_ERR_ALIGN;
+  const size_t need = bro_gemm_workspace_bytes(M, N, K);
+  if (need > 0 && (!workspace || workspace_bytes < need)) return BRO_ERR_WORKSPACE;
+  if (M == 0 || N == 0) return BRO_OK;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,
+                           workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,
+                      const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  if (!x_bf16 || !wcodes || !wscales || !y_bf16) return BRO_ERR_NULL;
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
+  if (M == 0 || N == 0) return BRO_OK;
+  if (!workspace) return BRO_ERR_NULL;
+  if (!aligned(workspace, 1024)) return BRO_ERR_ALIGN;
+  if (workspace_bytes < bro_linear_workspace_bytes(M, N, K)) return BRO_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* acodes = ws;
+  uint8_t* ascales = acodes + align_up(bro_codes_bytes(M, K), 1024);
+  uint8_t* gws = ascales + align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 1024);
+  bro_status rc = bro_rotate_quantize_mxfp4(x_bf16, M, K, ldx, block, acodes, ascales, BRO_LAYOUT_GEMM, stream);
+  if (rc != BRO_OK) return rc;
+  return bro_gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
+                        bro_gemm_workspace_bytes(M, N, K), stream);
+}
+
+bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block, const void* wcodes,
+                           const void* wscales, int64_t N, void* y_host_bf16, void* x_stage, void* y_stage,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  if (!x_host_bf16 || !y_host_bf16 || !x_stage || !y_stage) return BRO_ERR_NULL;
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
+  if (M == 0 || N == 0) return BRO_OK;
+  if (N % 8 != 0) return BRO_ERR_SHAPE;   // dense y staging needs a 16-byte row pitch
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return BRO_ERR_CUDA;
+  bro_status rc = bro_linear(x_stage, M, K, K, block, wcodes, wscales, N, y_stage, N, workspace,
+                             workspace_bytes, stream);
+  if (rc != BRO_OK) return rc;
+  if (cudaMemcpyAsync(y_host_bf16, y_stage, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return BRO_ERR_CUDA;
+  return BRO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,258 @@
+// Kernel 1: fused block-Hadamard rotation + MXFP4 quantisation (paper Sec. 4.3 Eq. 1, Sec. 4.1).
+//
+// HBM-bound streaming kernel: 2 bytes in and 0.53125 bytes out per element, one pass.
+//
+//  * One persistent CTA per SM.  A producer thread streams 128-row x 128-column bf16 tiles into
+//    a ring of shared-memory stages with TMA (two 128x64 boxes per tile, 128-byte swizzle), so
+//    the loads in flight are bounded by shared memory, not by registers.
+//  * 16 consumer warps.  Each thread owns one whole MX group (32 consecutive channels of one
+//    row): four conflict-free 16-byte shared loads, then the 5 butterfly stages of the 32-point
+//    Walsh-Hadamard transform entirely in registers — no shuffles for block = 32.  Blocks of 64
+//    and 128 add one or two cross-lane stages (the 2 or 4 groups of a block sit in lanes that
+//    differ in bit 0 / bit 3).
+//  * fp32 arithmetic in exactly this order: butterflies (a+b, a-b) with ascending stride, one
+//    multiply by c = fp32(1/sqrt(block)), amax over the group, shared exponent
+//    E = max(expfield(amax) - 2, 0) - 127, r = y * 2^-E, round-to-nearest-even to E2M1 with
+//    saturation.  The multiply by c and the exact scaling by 2^-E are merged into one multiply by
+//    c*2^-E whenever that product is a normal fp32 (bit-identical result); otherwise the two
+//    multiplies are done separately.
+//  * Output: one 16-byte store of 32 packed codes per thread; the 4 scale bytes of a row inside
+//    the tile are gathered with two shuffles and written as one 32-bit store.
+#pragma once
+
+#include "bro_common.cuh"
+
+namespace bro {
+namespace rq {
+
+constexpr int kTileRows = 128;
+constexpr int kTileCols = 128;              // 4 MX groups
+constexpr int kBoxCols = 64;                // one TMA box: 128 rows x 64 bf16 = 128 B per row
+constexpr int kBoxBytes = kTileRows * kBoxCols * 2;   // 16 KiB
+constexpr int kStageBytes = 2 * kBoxBytes;            // 32 KiB
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 16;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + 1 producer warp
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct Params {
+  int64_t M, K;
+  int64_t tiles_m, tiles_k;     // tiles_k covers the scale padding when layout == GEMM
+  uint8_t* codes;               // [M, K/2]
+  uint8_t* scales;
+  int64_t scale_kblocks;        // GEMM layout: 512-byte blocks per 128-row block
+  int layout;                   // bro_layout
+};
+
+__device__ __forceinline__ uint32_t pack_e2m1x8(float r0, float r1, float r2, float r3, float r4,
+                                                float r5, float r6, float r7) {
+  // cvt.rn.satfinite.e2m1x2.f32 d, a, b : a -> bits 4..7, b -> bits 0..3 (nearest even, +-6 clamp)
+  uint32_t w;
+  asm("{ .reg .b8 b0, b1, b2, b3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+      "mov.b32 %0, {b0, b1, b2, b3}; }"
+      : "=r"(w)
+      : "f"(r0), "f"(r1), "f"(r2), "f"(r3), "f"(r4), "f"(r5), "f"(r6), "f"(r7));
+  return w;
+}
+
+// c = fp32 nearest 1/sqrt(2^LOG2B)
+template <int LOG2B>
+__device__ __forceinline__ constexpr uint32_t norm_bits() {
+  // even exponent: exact power of two; odd: fp32(sqrt 2) = 0x3FB504F3 scaled by a power of two
+  return (LOG2B % 2 == 0) ? (uint32_t)(127 - LOG2B / 2) << 23
+                          : 0x3FB504F3u - ((uint32_t)((LOG2B + 1) / 2) << 23);
+}
+
+// Quantise the 32 fp32 values v (pre-normalisation: y = v*c) of one MX group.
+// Returns the scale byte; writes 4 code words.
+__device__ __forceinline__ uint32_t quantize_group(const float (&v)[32], uint32_t cbits,
+                                                   uint32_t (&w)[4]) {
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(v[i]));
+  const float c = __uint_as_float(cbits);
+  // amax of y: rounding is monotonic, so max_i fl(|v_i| c) = fl(max_i |v_i| * c)
+  const uint32_t ef = __float_as_uint(__fmul_rn(m, c)) >> 23;
+  const uint32_t s = ef > 2u ? ef - 2u : 0u;
+  if (ef >= 27u && ef <= 250u) {
+    // c * 2^-E is a normal fp32: one multiply, bit-identical to (v*c)*2^-E
+    const float c2 = __uint_as_float(cbits + ((127u - s) << 23));
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      w[j] = pack_e2m1x8(__fmul_rn(v[8 * j + 0], c2), __fmul_rn(v[8 * j + 1], c2),
+                         __fmul_rn(v[8 * j + 2], c2), __fmul_rn(v[8 * j + 3], c2),
+                         __fmul_rn(v[8 * j + 4], c2), __fmul_rn(v[8 * j + 5], c2),
+                         __fmul_rn(v[8 * j + 6], c2), __fmul_rn(v[8 * j + 7], c2));
+  } else {
+    const float p = __uint_as_float((254u - s) << 23);   // 2^-E, E = s - 127
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      w[j] = pack_e2m1x8(
+          __fmul_rn(__fmul_rn(v[8 * j + 0], c), p), __fmul_rn(__fmul_rn(v[8 * j + 1], c), p),
+          __fmul_rn(__fmul_rn(v[8 * j + 2], c), p), __fmul_rn(__fmul_rn(v[8 * j + 3], c), p),
+          __fmul_rn(__fmul_rn(v[8 * j + 4], c), p), __fmul_rn(__fmul_rn(v[8 * j + 5], c), p),
+          __fmul_rn(__fmul_rn(v[8 * j + 6], c), p), __fmul_rn(__fmul_rn(v[8 * j + 7], c), p));
+  }
+  return s;
+}
+
+// In-register 32-point transform, ascending stride, natural (Sylvester) order.
+__device__ __forceinline__ void fwht32(float (&v)[32]) {
+#pragma unroll
+  for (int h = 1; h < 32; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if ((i & h) == 0) {
+        const float a = v[i], b = v[i + h];
+        v[i] = __fadd_rn(a, b);
+        v[i + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+}
+
+// One butterfly stage across two lanes that hold the low / high half of the pairs.
+// low lane: a + b ; high lane: a - b = fma(own, -1, other) (exact, no extra rounding).
+__device__ __forceinline__ void cross_lane_stage(float (&v)[32], int lane_mask, bool is_high) {
+  const float sgn = is_high ? -1.f : 1.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], lane_mask);
+    v[i] = __fmaf_rn(v[i], sgn, o);
+  }
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float* v) {
+  v[0] = __uint_as_float(q.x << 16);
+  v[1] = __uint_as_float(q.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(q.y << 16);
+  v[3] = __uint_as_float(q.y & 0xFFFF0000u);
+  v[4] = __uint_as_float(q.z << 16);
+  v[5] = __uint_as_float(q.z & 0xFFFF0000u);
+  v[6] = __uint_as_float(q.w << 16);
+  v[7] = __uint_as_float(q.w & 0xFFFF0000u);
+}
+
+template <int LOG2B>
+__global__ void __launch_bounds__(kThreads, 1)
+rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle needs 1 KiB
+  const uint32_t bar_base = smem_base + kStages * kStageBytes;
+  // full[s] at bar_base + 8*s ; empty[s] at bar_base + 8*(kStages + s)
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_base + 8 * s, 1);
+      mbar_init(bar_base + 8 * (kStages + s), kConsumerWarps);
+    }
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  const int64_t total_tiles = p.tiles_m * p.tiles_k;
+
+  if (warp == kConsumerWarps) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmx);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int64_t issued = 0;
+      for (int64_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int64_t tm = t / p.tiles_k, tk = t - tm * p.tiles_k;
+        if (issued >= kStages)
+          ok = mbar_wait(bar_base + 8 * (kStages + stage), phase ^ 1u, SITE_RQ_EMPTY);
+        if (!ok) break;
+        const uint32_t full = bar_base + 8 * stage;
+        const uint32_t dst = smem_base + stage * kStageBytes;
+        mbar_arrive_expect_tx(full, kStageBytes);
+        tma_load_2d(dst, &tmx, (int)(tk * kTileCols), (int)(tm * kTileRows), full);
+        tma_load_2d(dst + kBoxBytes, &tmx, (int)(tk * kTileCols + kBoxCols),
+                    (int)(tm * kTileRows), full);
+        ++issued;
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        // A consumer gave up.  Do not leave the CTA while copies may still land in its shared
+        // memory: wait (bounded) for the last load armed on every stage.  Issue i used stage
+        // i % kStages in phase (i / kStages) & 1.
+        const int64_t first = issued > kStages ? issued - kStages : 0;
+        for (int64_t i = first; i < issued; ++i)
+          mbar_wait(bar_base + 8 * (int)(i % kStages), (uint32_t)((i / kStages) & 1), SITE_RQ_DRAIN);
+      }
+    }
+  } else {
+    // ---------------- consumers ----------------
+    const int gg = lane & 1;                 // group within the 64-column box
+    const int box = (lane >> 3) & 1;         // which box of the tile
+    const int row = warp * 8 + ((lane >> 4) << 2) + ((lane >> 1) & 3);   // row within the tile
+    const int g = box * 2 + gg;              // group within the tile (0..3)
+    // 16-byte chunk j of this group sits at chunk index (gg*4 + j) ^ (row & 7) of its 128-B row
+    const uint32_t row_off = (uint32_t)box * kBoxBytes + (uint32_t)row * 128u;
+    const uint32_t sw = (uint32_t)(row & 7);
+    constexpr uint32_t cbits = norm_bits<LOG2B>();
+
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int64_t t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      const int64_t tm = t / p.tiles_k, tk = t - tm * p.tiles_k;
+      if (!mbar_wait(bar_base + 8 * stage, phase, SITE_RQ_FULL)) break;
+      const uint32_t src = smem_base + stage * kStageBytes + row_off;
+      float v[32];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint4 q = lds128(src + ((((uint32_t)gg * 4u + j) ^ sw) << 4));
+        unpack_bf16x8(q, v + 8 * j);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_base + 8 * (kStages + stage));
+      if (++stage == kStages) { stage = 0; phase ^= 1u; }
+
+      fwht32(v);
+      if (LOG2B >= 6) cross_lane_stage(v, 1, gg != 0);
+      if (LOG2B >= 7) cross_lane_stage(v, 8, box != 0);
+
+      uint32_t w[4];
+      const uint32_t s = quantize_group(v, cbits, w);
+
+      const int64_t grow = tm * kTileRows + row;
+      const int64_t ggrp = tk * (kTileCols / 32) + g;     // group index along K
+      const bool in_k = ggrp * 32 < p.K;
+      if (grow < p.M && in_k) {
+        uint4* dst = reinterpret_cast<uint4*>(p.codes + grow * (p.K >> 1) + ggrp * 16);
+        *dst = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      // gather the row's 4 scale bytes of this tile into the lane with gg == 0 && box == 0
+      uint32_t sb = in_k ? s : 0u;
+      sb |= __shfl_xor_sync(0xFFFFFFFFu, sb, 1) << 8;
+      sb |= __shfl_xor_sync(0xFFFFFFFFu, sb, 8) << 16;
+      if (g == 0) {
+        if (p.layout == BRO_LAYOUT_GEMM) {
+          // 512-byte block (tm, tk): byte (r%32)*16 + (r/32)*4 + g ; padding rows included
+          const int64_t off = (tm * p.scale_kblocks + tk) * 512 + (row & 31) * 16 + (row >> 5) * 4;
+          *reinterpret_cast<uint32_t*>(p.scales + off) = sb;
+        } else if (grow < p.M) {
+          const int64_t ng = p.K >> 5;
+          uint8_t* dst = p.scales + grow * ng + tk * 4;
+          if (tk * 4 + 4 <= ng && ((reinterpret_cast<uintptr_t>(dst) & 3) == 0)) {
+            *reinterpret_cast<uint32_t*>(dst) = sb;
+          } else {
+            for (int i = 0; i < 4 && tk * 4 + i < ng; ++i) dst[i] = (uint8_t)(sb >> (8 * i));
+          }
+        }
+      }
+    }
+  }
+}
+
+}  // namespace rq
+}  // namespace bro
