@@ -68,6 +68,10 @@ typedef enum { BRO_OUT_BF16 = 0, BRO_OUT_F32 = 1 } bro_out_dtype;
 /* Human-readable name of a status code (static string, never NULL). */
 const char* bro_status_string(bro_status s);
 
+/* Text of the most recent CUDA runtime/driver error this thread saw inside a libbro call that
+ * returned BRO_ERR_CUDA ("" if none).  Static storage; valid until the next libbro call. */
+const char* bro_last_cuda_error(void);
+
 /* rows*K/2: bytes of a packed code tensor. */
 size_t bro_codes_bytes(int64_t rows, int64_t K);
 /* Bytes of a scale tensor in the given layout (padded for BRO_LAYOUT_GEMM). 0 on bad input. */

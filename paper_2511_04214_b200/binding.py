@@ -21,7 +21,7 @@ OUT_BF16 = 0
 OUT_F32 = 1
 
 EXPORTS = [
-    "bro_status_string", "bro_codes_bytes", "bro_scales_bytes", "bro_scale_offset",
+    "bro_status_string", "bro_last_cuda_error", "bro_codes_bytes", "bro_scales_bytes", "bro_scale_offset",
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host",
@@ -31,7 +31,8 @@ EXPORTS = [
 class BroError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = int(code)
-        super().__init__(f"{where}: {status_string(code)} ({code})")
+        detail = lib.bro_last_cuda_error().decode() if int(code) == 6 else ""
+        super().__init__(f"{where}: {status_string(code)} ({code}) {detail}".rstrip())
 
 
 def _load() -> ctypes.CDLL:
@@ -43,6 +44,8 @@ def _load() -> ctypes.CDLL:
     i64, p, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
     L.bro_status_string.restype = ctypes.c_char_p
     L.bro_status_string.argtypes = [ci]
+    L.bro_last_cuda_error.restype = ctypes.c_char_p
+    L.bro_last_cuda_error.argtypes = []
     L.bro_codes_bytes.restype = sz
     L.bro_codes_bytes.argtypes = [i64, i64]
     L.bro_scales_bytes.restype = sz

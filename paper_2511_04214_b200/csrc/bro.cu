@@ -70,7 +70,10 @@ bro_status make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t elem_byt
                        uint64_t inner, uint64_t rows, uint64_t pitch_bytes, uint32_t box_inner,
                        uint32_t box_rows, CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return BRO_ERR_CUDA;
+  if (!fn) {
+    snprintf(bro::g_last_cuda_error, sizeof(bro::g_last_cuda_error), "cuTensorMapEncodeTiled unavailable");
+    return BRO_ERR_CUDA;
+  }
   cuuint64_t dims[2] = {inner, rows};
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {box_inner, box_rows};
@@ -79,24 +82,38 @@ bro_status make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, size_t elem_byt
   CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    snprintf(bro::g_last_cuda_error, sizeof(bro::g_last_cuda_error), "cuTensorMapEncodeTiled: CUresult %d", (int)r);
   return r == CUDA_SUCCESS ? BRO_OK : BRO_ERR_CUDA;
 }
 
 template <typename K>
 bro_status set_smem(K kernel, int bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
+  return bro::cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes),
+                      "cudaFuncSetAttribute")
              ? BRO_OK
              : BRO_ERR_CUDA;
 }
 
 int64_t gemm_scale_kblocks(int64_t K) { return 2 * ceil_div(K, 256); }
 
+}  // namespace
+
+// Packed 4-bit codes viewed as bytes: [rows, K/2], box = 128 bytes x box_rows, 128-byte swizzle.
+bro_status bro::gemm::make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows) {
+  return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, base, (uint64_t)(K / 2), (uint64_t)rows,
+                     (uint64_t)(K / 2), 128, (uint32_t)box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+namespace {
+
 // ---- rotate + quantise ---------------------------------------------------------------------------
 bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, int block,
                                   void* codes, void* scales, bro_layout layout, cudaStream_t st) {
-  if (!x || !codes || !scales) return BRO_ERR_NULL;
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (M == 0 && (layout == BRO_LAYOUT_CANONICAL || layout == BRO_LAYOUT_GEMM)) return BRO_OK;
+  if (!x || !codes || !scales) return BRO_ERR_NULL;
   if (layout != BRO_LAYOUT_CANONICAL && layout != BRO_LAYOUT_GEMM) return BRO_ERR_SHAPE;
   const int64_t B = block == 0 ? K : block;
   if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
@@ -129,22 +146,24 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   const int64_t tiles = p.tiles_m * p.tiles_k;
   const int grid = (int)(tiles < di.sm_count ? tiles : di.sm_count);
 
-  auto go = [&](auto kernel) -> bro_status {
-    static thread_local bool attr_done[64] = {};
+  // (All three instantiations share one function-pointer type, so the opt-in to large dynamic
+  // shared memory is keyed by the kernel's address, per device.)
+  auto go = [&](void (*kernel)(CUtensorMap, Params), int which) -> bro_status {
+    static bool attr_done[64][3] = {};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (!attr_done[dev]) {
+    if (!attr_done[dev][which]) {
       bro_status r = set_smem(kernel, bro::rq::kSmemBytes);
       if (r != BRO_OK) return r;
-      attr_done[dev] = true;
+      attr_done[dev][which] = true;
     }
     kernel<<<grid, bro::rq::kThreads, bro::rq::kSmemBytes, st>>>(tmx, p);
-    return cudaGetLastError() == cudaSuccess ? BRO_OK : BRO_ERR_CUDA;
+    return bro::cuda_ok(cudaGetLastError(), "rotate_quantize launch") ? BRO_OK : BRO_ERR_CUDA;
   };
   switch (B) {
-    case 32: return go(bro::rq::rotate_quantize_kernel<5>);
-    case 64: return go(bro::rq::rotate_quantize_kernel<6>);
-    default: return go(bro::rq::rotate_quantize_kernel<7>);
+    case 32: return go(bro::rq::rotate_quantize_kernel<5>, 0);
+    case 64: return go(bro::rq::rotate_quantize_kernel<6>, 1);
+    default: return go(bro::rq::rotate_quantize_kernel<7>, 2);
   }
 }
 
@@ -152,6 +171,8 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
 
 // =================================================================================================
 extern "C" {
+
+const char* bro_last_cuda_error(void) { return bro::g_last_cuda_error; }
 
 const char* bro_status_string(bro_status s) {
   switch (s) {
@@ -225,10 +246,11 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
                           const void* wscales, int64_t M, int64_t N, int64_t K, void* y, int64_t ldy,
                           bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
                           void* stream) {
-  if (!acodes || !ascales || !wcodes || !wscales || !y) return BRO_ERR_NULL;
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0 || ldy < N) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (out_dtype != BRO_OUT_BF16 && out_dtype != BRO_OUT_F32) return BRO_ERR_SHAPE;
+  if (M == 0 || N == 0) return BRO_OK;
+  if (!acodes || !ascales || !wcodes || !wscales || !y) return BRO_ERR_NULL;
   const int64_t esz = out_dtype == BRO_OUT_BF16 ? 2 : 4;
   if (!aligned(acodes, 128) || !aligned(wcodes, 128) || !aligned(ascales, 128) || !aligned(wscales, 128) ||
       !aligned(y, 16) || (ldy * esz) % 16 != 0)
@@ -246,10 +268,9 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
 bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,
                       const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
                       size_t workspace_bytes, void* stream) {
-  if (!x_bf16 || !wcodes || !wscales || !y_bf16) return BRO_ERR_NULL;
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
   if (M == 0 || N == 0) return BRO_OK;
-  if (!workspace) return BRO_ERR_NULL;
+  if (!x_bf16 || !wcodes || !wscales || !y_bf16 || !workspace) return BRO_ERR_NULL;
   if (!aligned(workspace, 1024)) return BRO_ERR_ALIGN;
   if (workspace_bytes < bro_linear_workspace_bytes(M, N, K)) return BRO_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -265,9 +286,9 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
 bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block, const void* wcodes,
                            const void* wscales, int64_t N, void* y_host_bf16, void* x_stage, void* y_stage,
                            void* workspace, size_t workspace_bytes, void* stream) {
-  if (!x_host_bf16 || !y_host_bf16 || !x_stage || !y_stage) return BRO_ERR_NULL;
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
   if (M == 0 || N == 0) return BRO_OK;
+  if (!x_host_bf16 || !y_host_bf16 || !x_stage || !y_stage) return BRO_ERR_NULL;
   if (N % 8 != 0) return BRO_ERR_SHAPE;   // dense y staging needs a 16-byte row pitch
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(x_stage, x_host_bf16, (size_t)M * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)

@@ -5,10 +5,19 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include "../../include/bro.h"
 
 namespace bro {
+
+// Host side: remember the text of the last failing CUDA call of this thread.
+inline thread_local char g_last_cuda_error[256] = "";
+inline bool cuda_ok(cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return true;
+  snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return false;
+}
 
 // One status word per device (each device that loads the module gets its own instance).
 // 0 = OK; otherwise (BRO_ERR_TIMEOUT) | (site << 8).  Kernels only ever move it away from 0.

@@ -1,12 +1,328 @@
-// Kernel 2 placeholder: replaced by the tcgen05 block-scaled GEMM.
+// Kernel 2: block-scaled MXFP4 x MXFP4 GEMM on the 5th-generation tensor cores
+// (paper Sec. 1 / Sec. 4.2: W4A4, y = Q(xR) Q(WR)^T; fp32 accumulation, bf16 or fp32 output).
+//
+//   y[m, n] = sum_g 2^(Ea[m,g] + Ew[n,g]) * sum_{k in g} a[m,k] w[n,k]
+//
+// One CTA computes a 128 x BN output tile.  Warp-specialised:
+//   warp 0      TMA producer: per 256-element K step, one 128x128-byte box of A codes, one
+//               BNx128-byte box of W codes (128-byte swizzle) and the matching 512-byte scale
+//               blocks (plain bulk copies; the scale tensors are already in tensor-core order).
+//   warp 1      owns TMEM; one elected thread copies the scale blocks shared -> TMEM
+//               (tcgen05.cp) and issues four tcgen05.mma kind::mxf4.block_scale (K = 64 each)
+//               per K step into a 128 x BN fp32 accumulator in TMEM; tcgen05.commit releases the
+//               shared-memory stage and finally signals the epilogue.
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (one TMEM lane quadrant per warp), convert,
+//               store.
+// Every mbarrier wait is bounded; on expiry the role records the site and falls through to the
+// common exit, where TMEM is released.
 #pragma once
+
+#include <stdlib.h>
+
 #include "bro_common.cuh"
+
 namespace bro {
 namespace gemm {
-inline size_t workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
-inline bro_status launch(const void*, const void*, const void*, const void*, int64_t, int64_t, int64_t,
-                         void*, int64_t, int, void*, size_t, int, cudaStream_t) {
-  return BRO_ERR_UNSUPPORTED;
+
+constexpr int kBM = 128;
+constexpr int kBK = 256;                    // elements per K step = 128 bytes of codes per row
+constexpr int kThreads = 192;
+constexpr int kATileBytes = kBM * 128;      // 16 KiB
+
+template <int BN> struct Cfg {
+  static constexpr int kStages = BN == 256 ? 4 : 3;
+  static constexpr int kBTileBytes = BN * 128;
+  static constexpr int kSfaBytes = 1024;                  // 2 blocks of 512 B (128 rows x 4 groups)
+  static constexpr int kSfbBytes = (BN / 128) * 1024;
+  static constexpr int kStageBytes = kATileBytes + kBTileBytes + kSfaBytes + kSfbBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int kSfaCols = 8;                      // 2 K-blocks x 4 columns
+  static constexpr int kSfbCols = (BN / 32) * 2;          // 2 K-blocks x BN/32 columns
+  static constexpr int kTmemCols = BN == 256 ? 512 : 256; // power of two >= BN + SF columns
+};
+
+struct Params {
+  const uint8_t* ascales;
+  const uint8_t* wscales;
+  void* y;
+  int64_t M, N, K, ldy;
+  int64_t kblocks;          // 512-byte scale blocks per 128-row block = 2*ceil(K/256)
+  int num_k_steps;          // ceil(K/256)
+};
+
+// ---- tcgen05 wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+               : "memory");
 }
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p; }" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- descriptors -------------------------------------------------------------------------------
+// Shared-memory matrix descriptor, K-major operand stored as rows of 128 bytes with the 128-byte
+// swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);   // start address / 16
+  d |= (uint64_t)1 << 16;                   // leading byte offset / 16 (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset / 16
+  d |= (uint64_t)1 << 46;                   // descriptor version (sm_100)
+  d |= (uint64_t)2 << 61;                   // layout: 128-byte swizzle
+  return d;
+}
+// Scale block: 32 rows x 16 bytes, dense, no swizzle; 8-row groups 128 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sf(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)(128 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+// Instruction descriptor, kind::mxf4 block-scaled: E2M1 x E2M1, both K-major, UE8M0 scales,
+// dense K = 64, M x N = 128 x BN; scale-factor byte ids filled in per K block.
+template <int BN>
+__device__ __forceinline__ constexpr uint32_t make_idesc() {
+  return (1u << 7) /*A = E2M1*/ | (1u << 10) /*B = E2M1*/ | ((uint32_t)(BN >> 3) << 17) | (1u << 23) /*UE8M0*/ |
+         ((uint32_t)(kBM >> 4) << 24);
+}
+
+template <int BN, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw, const Params p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sA = smem_base;
+  const uint32_t sB = sA + C::kStages * kATileBytes;
+  const uint32_t sSFA = sB + C::kStages * C::kBTileBytes;
+  const uint32_t sSFB = sSFA + C::kStages * C::kSfaBytes;
+  const uint32_t bar_base = sSFB + C::kStages * C::kSfbBytes;
+  const uint32_t bar_full = bar_base;                       // [kStages]
+  const uint32_t bar_empty = bar_base + 8 * C::kStages;     // [kStages]
+  const uint32_t bar_acc = bar_base + 16 * C::kStages;      // accumulator ready
+  const uint32_t tmem_slot = bar_acc + 8;                   // u32 written by tcgen05.alloc
+  uint32_t* tmem_slot_ptr =
+      reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t m0 = (int64_t)blockIdx.y * kBM;
+  const int64_t n0 = (int64_t)blockIdx.x * BN;
+  const int nblk_valid = (n0 + 128 < p.N && BN == 256) ? 2 : 1;   // 128-row scale blocks of W in range
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    mbar_init(bar_acc, 1);
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  const uint32_t tmem_acc = tmem_base;
+  const uint32_t tmem_sfa = tmem_base + BN;
+  const uint32_t tmem_sfb = tmem_base + BN + C::kSfaCols;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tma);
+      tma_prefetch_desc(&tmw);
+      int stage = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      bool ok = true;
+      const uint8_t* sfa_src = p.ascales + (int64_t)blockIdx.y * p.kblocks * 512;
+      const uint8_t* sfb_src = p.wscales + (n0 / 128) * p.kblocks * 512;
+      for (int ks = 0; ks < p.num_k_steps; ++ks) {
+        if (issued >= C::kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
+        if (!ok) break;
+        const uint32_t full = bar_full + 8 * stage;
+        mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
+        tma_load_2d(sA + stage * kATileBytes, &tma, ks * 128, (int)m0, full);
+        tma_load_2d(sB + stage * C::kBTileBytes, &tmw, ks * 128, (int)n0, full);
+        bulk_load_1d(sSFA + stage * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
+        for (int nb = 0; nb < nblk_valid; ++nb)
+          bulk_load_1d(sSFB + stage * C::kSfbBytes + nb * 1024,
+                       sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512, 1024, full);
+        ++issued;
+        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        const int first = issued > C::kStages ? issued - C::kStages : 0;
+        for (int i = first; i < issued; ++i)
+          mbar_wait(bar_full + 8 * (i % C::kStages), (uint32_t)((i / C::kStages) & 1), SITE_GEMM_DRAIN);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc0 = make_idesc<BN>();
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int ks = 0; ks < p.num_k_steps && ok; ++ks) {
+        ok = mbar_wait(bar_full + 8 * stage, phase, SITE_GEMM_FULL);
+        if (!ok) break;
+        tc_fence_after();
+        // scale blocks of this K step: shared -> TMEM.  K-block pair a (128 elements) of A goes to
+        // columns 4a..4a+3; of W to columns (BN/32)*a + 4*nb .. +3.
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+          tc_cp_sf(tmem_sfa + 4 * a, smem_desc_sf(sSFA + stage * C::kSfaBytes + a * 512));
+#pragma unroll
+          for (int nb = 0; nb < BN / 128; ++nb)
+            tc_cp_sf(tmem_sfb + (BN / 32) * a + 4 * nb,
+                     smem_desc_sf(sSFB + stage * C::kSfbBytes + nb * 1024 + a * 512));
+        }
+        const uint64_t adesc = smem_desc_sw128(sA + stage * kATileBytes);
+        const uint64_t bdesc = smem_desc_sw128(sB + stage * C::kBTileBytes);
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint32_t sf_id = (kb & 1) * 2;            // bytes {0,1} or {2,3} of the scale word
+          const uint32_t idesc = idesc0 | (sf_id << 4) | (sf_id << 29);
+          const uint32_t tsfa = (tmem_sfa + 4 * (kb >> 1)) | (sf_id << 30);
+          const uint32_t tsfb = (tmem_sfb + (BN / 32) * (kb >> 1)) | (sf_id << 30);
+          tc_mma_mxf4(tmem_acc, adesc + 2 * kb, bdesc + 2 * kb, idesc, tsfa, tsfb, (ks | kb) != 0 ? 1u : 0u);
+        }
+        tc_commit(bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
+        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+      }
+      tc_commit(bar_acc);                   // accumulator complete (or abandoned) -> epilogue
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    const bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc, 0, SITE_GEMM_ACC_FULL));
+    tc_fence_after();
+    const int64_t row = m0 + q * 32 + lane;
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tc_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
+        tc_wait_ld();
+        const int64_t col0 = n0 + c * 32;
+        if (row < p.M && col0 < p.N) {
+          if (OUT_F32) {
+            float* dst = static_cast<float*>(p.y) + row * p.ldy + col0;
+            if (col0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                reinterpret_cast<uint4*>(dst)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+            } else {
+              for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __uint_as_float(r[j]);
+            }
+          } else {
+            uint16_t* dst = static_cast<uint16_t*>(p.y) + row * p.ldy + col0;
+            uint32_t h[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r[2 * j + 1])), "f"(__uint_as_float(r[2 * j])));
+            if (col0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                reinterpret_cast<uint4*>(dst)[j] = make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+            } else {
+              for (int j = 0; j < 32 && col0 + j < p.N; ++j)
+                dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFF));
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+inline size_t workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+
+bro_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows);
+
+template <int BN>
+bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const Params& p, int out_dtype,
+                       cudaStream_t st) {
+  using C = Cfg<BN>;
+  dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + kBM - 1) / kBM));
+  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
+    static bool attr_done[64][2] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_done[dev][which]) {
+      if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes),
+                   "cudaFuncSetAttribute(gemm)"))
+        return BRO_ERR_CUDA;
+      attr_done[dev][which] = true;
+    }
+    kernel<<<grid, kThreads, C::kSmemBytes, st>>>(tma, tmw, p);
+    return cuda_ok(cudaGetLastError(), "gemm_mxfp4 launch") ? BRO_OK : BRO_ERR_CUDA;
+  };
+  return out_dtype == BRO_OUT_F32 ? go(gemm_mxfp4_kernel<BN, true>, 1) : go(gemm_mxfp4_kernel<BN, false>, 0);
+}
+
+inline bro_status launch(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
+                         int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* /*ws*/,
+                         size_t /*ws_bytes*/, int /*sm_count*/, cudaStream_t st) {
+  if ((M + kBM - 1) / kBM > 65535) return BRO_ERR_UNSUPPORTED;
+  int bn = 256;
+  if (const char* e = getenv("BRO_GEMM_TILE_N")) bn = atoi(e) == 128 ? 128 : 256;
+  else if (N <= 128) bn = 128;
+  Params p;
+  p.ascales = static_cast<const uint8_t*>(ascales);
+  p.wscales = static_cast<const uint8_t*>(wscales);
+  p.y = y;
+  p.M = M; p.N = N; p.K = K; p.ldy = ldy;
+  p.num_k_steps = (int)((K + kBK - 1) / kBK);
+  p.kblocks = 2 * (int64_t)p.num_k_steps;
+  CUtensorMap tma, tmw;
+  bro_status rc = make_codes_map(&tma, acodes, M, K, kBM);
+  if (rc != BRO_OK) return rc;
+  rc = make_codes_map(&tmw, wcodes, N, K, bn);
+  if (rc != BRO_OK) return rc;
+  return bn == 256 ? launch_tile<256>(tma, tmw, p, out_dtype, st) : launch_tile<128>(tma, tmw, p, out_dtype, st);
+}
+
 }  // namespace gemm
 }  // namespace bro

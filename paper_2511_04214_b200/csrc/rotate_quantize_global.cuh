@@ -127,7 +127,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, void*
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return BRO_ERR_CUDA;
     kernel<<<grid, threads, smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? BRO_OK : BRO_ERR_CUDA;
+    return cuda_ok(cudaGetLastError(), "rotate_quantize_global launch") ? BRO_OK : BRO_ERR_CUDA;
   };
   if (threads <= 256) return go(rotate_quantize_global_kernel<256>);
   if (threads <= 512) return go(rotate_quantize_global_kernel<512>);

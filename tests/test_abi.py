@@ -87,6 +87,7 @@ def test_argument_validation_needs_no_device(lib):
     assert L.bro_rotate_quantize_mxfp4(p(a16), 0, 64, 64, 32, p(a16), p(a16), 0, None) == 0
     a128 = (a + 127) // 128 * 128
     assert L.bro_gemm_mxfp4(p(a128), p(a128), p(a128), None, 1, 8, 32, p(a128), 8, 0, None, 0, None) == 1
+    assert L.bro_gemm_mxfp4(None, None, None, None, 0, 8, 32, None, 8, 0, None, 0, None) == 0
     assert L.bro_gemm_mxfp4(p(a128), p(a128), p(a128), p(a128), 1, 8, 40, p(a128), 8, 0, None, 0, None) == 2
     assert L.bro_gemm_mxfp4(p(a128), p(a128), p(a128), p(a128), 1, 8, 32, p(a128), 4, 0, None, 0, None) == 2
     assert L.bro_gemm_mxfp4(p(a128 + 16), p(a128), p(a128), p(a128), 1, 8, 32, p(a128), 8, 0, None, 0, None) == 3
