@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the block-rotated MXFP4 W4A4 linear layer on B200.
+
+One *step* = one pass of the whole hot path — fused block-Hadamard rotation + MXFP4 quantisation
+of the activations, then the block-scaled MXFP4 GEMM against pre-packed weights — over every
+shape of the workload (default: the three LLaMA-3.2-1B-shaped layers, M = 2048 tokens).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg5] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is device-timed throughput with inputs resident in HBM;
+`e2e` is the same metric through the host-buffer entry point (H2D of x and D2H of y inside the
+timed region); `roofline` describes the dominant kernel (the GEMM) timed per launch with CUDA
+events; `cpu_baseline` is the CPU oracle on a bounded sample.  With --gpus N > 1 (launched by
+torchrun) every rank runs an independent replica — the path has no cross-GPU exchange.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "MXFP4 W4A4 linear TFLOPS (rotate+quantize+GEMM)"
+UNIT = "TFLOP/s"
+L2_BYTES = 126 * 1024 * 1024
+FP4_OVER_BF16 = 4.0          # nominal dense fp4 : bf16 tensor throughput ratio on B200 (9 : 2.25)
+
+
+def workload_shapes(name):
+    from paper_2511_04214_b200 import synth
+    cfg = synth.CONFIGS[name]
+    shapes = [s for s in cfg["shapes"] if s[2] > 0]
+    return cfg, shapes
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the GPU works."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.marks = {}
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def mark(self, name):
+        self.marks[name] = time.time()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        t0, t1 = self.marks.get("t0", 0), self.marks.get("t1", float("inf"))
+        inside, allc, smax, reasons, power = [], [], None, set(), []
+        for (t, line) in self.rows:
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm, mx = float(f[1]), float(f[2])
+            except ValueError:
+                continue
+            smax = mx
+            allc.append(sm)
+            if t0 <= t <= t1 + 0.1:
+                inside.append(sm)
+                try:
+                    power.append(float(f[3]))
+                except ValueError:
+                    pass
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        use = inside if inside else allc
+        return {"sm_mhz": statistics.median(use) if use else None, "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples_in_timed_region": len(inside),
+                "power_w_max": max(power) if power else None}
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_prepare(shapes, cfg, rows_per_shape, block):
+    """Inputs for the CPU oracle: the first `rows_per_shape` rows of every shape, weights packed by
+    the oracle (offline, untimed)."""
+    import oracle
+    from paper_2511_04214_b200 import synth
+    prepared = []
+    for i, (M, K, N) in enumerate(shapes):
+        m = min(M, rows_per_shape)
+        x = synth.activations(m, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
+        w = synth.weights(N, K, seed=cfg["seed"] + i)
+        wc, ws = oracle.pack_weights(synth.bf16_bits(w), block)
+        prepared.append((synth.bf16_bits(x), wc, ws, m, K, N))
+    return prepared
+
+
+def oracle_step(prepared, block):
+    """One pass of the oracle's whole layer over the prepared sample.  Returns (seconds, flops)."""
+    import oracle
+    t0 = time.perf_counter()
+    flops = 0.0
+    for (xb, wc, ws, m, K, N) in prepared:
+        oracle.linear(xb, block, wc, ws)
+        flops += 2.0 * m * K * N
+    return time.perf_counter() - t0, flops
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload,
+    sized so that warmup + steps finish in about two minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfg, shapes = workload_shapes(args.workload)
+    rows = args.ref_rows
+    if rows <= 0:
+        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block), args.block)
+        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block), args.block)
+        rows = int(max(1, min(64, 120.0 / (max(args.steps + args.warmup, 1) * max(t1, 1e-4)))))
+    prepared = oracle_prepare(shapes, cfg, rows, args.block)
+    for _ in range(max(args.warmup, 0)):
+        oracle_step(prepared, args.block)
+    total_t, total_f = 0.0, 0.0
+    for _ in range(args.steps):
+        t, f = oracle_step(prepared, args.block)
+        total_t += t
+        total_f += f
+    value = total_f / total_t / 1e12
+    sample = f"first {rows} rows of each of {len(shapes)} shapes per step (weights packed offline, untimed)"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_t / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": args.workload, "shapes_MKN": shapes, "block": args.block,
+                                         "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2511_04214_b200 import build
+    build.build()
+    from paper_2511_04214_b200 import binding as bro, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+    dev = torch.device("cuda", local_rank)
+    cfg, shapes = workload_shapes(args.workload)
+    block = args.block
+    peaks = measured_peaks()
+
+    # ---- inputs: a ring of independent activation/output sets so that consecutive steps never
+    # find their inputs in L2 (126 MB).
+    per_step_bytes = sum(M * K * 2 + N * K // 2 + M * N * 2 for (M, K, N) in shapes)
+    ring = max(2, min(8, -(-3 * L2_BYTES // per_step_bytes)))
+    sets = []
+    stream = torch.cuda.current_stream()
+    for i, (M, K, N) in enumerate(shapes):
+        w = synth.weights(N, K, seed=cfg["seed"] + i).to(dev)
+        x0 = synth.activations(M, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
+        ws_bytes = bro.linear_workspace_bytes(M, N, K)
+        per_ring = []
+        for r in range(ring):
+            wcodes = bro.alloc_codes(N, K, dev)
+            wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM, dev)
+            bro.pack_weights(w, block, wcodes, wscales)                  # offline, untimed
+            x = x0.to(dev).roll(r * 7, 0).contiguous()        # same statistics, separate memory
+            per_ring.append({"x": x, "wcodes": wcodes, "wscales": wscales,
+                             "y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+                             "ws": bro.alloc_workspace(ws_bytes, dev)})
+        sets.append(per_ring)
+        del w
+    torch.cuda.synchronize()
+
+    def step(r):
+        for i, (M, K, N) in enumerate(shapes):
+            s = sets[i][r % ring]
+            bro.linear(s["x"], block, s["wcodes"], s["wscales"], N, s["y"], s["ws"])
+
+    flops_per_step = sum(2.0 * M * K * N for (M, K, N) in shapes)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    # ---- warm-up (also sets kernel attributes before any graph capture)
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+
+    graph = None
+    if not args.no_graph:
+        # One CUDA graph = `ring` consecutive steps; replayed steps/ring times.
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for r in range(ring):
+                step(r)
+        graph.replay()
+        torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    steps = args.steps
+    if graph is not None:
+        replays = max(1, -(-steps // ring))
+        steps = replays * ring
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark("t0")
+    e0.record()
+    if graph is not None:
+        for _ in range(replays):
+            graph.replay()
+    else:
+        for i in range(steps):
+            step(i)
+    e1.record()
+    barrier()
+    sampler.mark("t1")
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    status = bro.last_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {bro.status_string(status)} after the timed region")
+    value = flops_per_step * steps * world / (ms_total * 1e-3) / 1e12
+
+    # ---- instrumented pass: the same launches with an event after every kernel (rotate+quantize
+    # and GEMM issued as the two C-ABI calls bro_linear makes), for the per-kernel roofline.
+    inst_steps = min(steps, 40)
+    rq_ms = [[] for _ in shapes]
+    gemm_ms = [[] for _ in shapes]
+    for it in range(inst_steps + 3):
+        for i, (M, K, N) in enumerate(shapes):
+            s = sets[i][it % ring]
+            acodes = s["ws"][:bro.codes_bytes(M, K)]
+            off = (bro.codes_bytes(M, K) + 1023) // 1024 * 1024
+            ascales = s["ws"][off:off + bro.scales_bytes(M, K, bro.LAYOUT_GEMM)]
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
+            ev[1].record()
+            bro.gemm_mxfp4(acodes, ascales, s["wcodes"], s["wscales"], M, N, K, s["y"])
+            ev[2].record()
+            if it >= 3:
+                rq_ms[i].append((ev[0], ev[1]))
+                gemm_ms[i].append((ev[1], ev[2]))
+    torch.cuda.synchronize()
+    rq_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) for lst in rq_ms]
+    gemm_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) for lst in gemm_ms]
+    gemm_flops = sum(2.0 * M * K * N for (M, K, N) in shapes)
+    gemm_tflops = gemm_flops / (sum(gemm_t) * 1e-3) / 1e12
+    rq_bytes = sum(M * K * 2.53125 for (M, K, N) in shapes)
+    rq_gbs = rq_bytes / (sum(rq_t) * 1e-3) / 1e9
+    fp4_peak = peaks["bf16_tflops"] * FP4_OVER_BF16
+    gemm_bytes = sum((M + N) * K * (0.5 + 1 / 32) + 2 * M * N for (M, K, N) in shapes)
+
+    # ---- end-to-end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        for i, (M, K, N) in enumerate(shapes):
+            s = sets[i][0]
+            host.append({"xh": s["x"].cpu().pin_memory(),
+                         "yh": torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
+                         "xs": torch.empty((M, K), dtype=torch.bfloat16, device=dev)})
+
+        def e2e_step():
+            for i, (M, K, N) in enumerate(shapes):
+                s, h = sets[i][0], host[i]
+                bro.linear_host(h["xh"], block, s["wcodes"], s["wscales"], N, h["yh"], h["xs"], s["y"], s["ws"])
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        n_e2e = max(3, min(steps, 30))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        barrier()
+        ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": flops_per_step * n_e2e * world / (ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": sum(M * K * 2 for (M, K, N) in shapes),
+               "d2h_bytes_per_step": sum(M * N * 2 for (M, K, N) in shapes), "steps": n_e2e}
+
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        t_probe, f_probe = oracle_step(oracle_prepare(shapes, cfg, 8, block), block)
+        rows = int(max(8, min(512, 8 * 12.0 / max(t_probe, 1e-3))))
+        t, f = oracle_step(oracle_prepare(shapes, cfg, rows, block), block)
+        cpu = {"value": f / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"first {rows} rows of each of the {len(shapes)} shapes, {t:.1f} s (weights packed offline, untimed)"}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "mxfp4 (e2m1 x e8m0) operands, f32 accumulate, bf16 out", "data": "synthetic",
+            "config": {"workload": args.workload, "shapes_MKN": shapes, "block": block,
+                       "l2": f"ring of {ring} independent input/output sets ({per_step_bytes * ring / 1e6:.0f} MB) > 126 MB L2",
+                       "launch": "cuda_graph" if graph is not None else "direct", "parallelism": "replicas only"},
+            "clocks": clocks,
+            "e2e": e2e,
+            "gpu_launches": steps * len(shapes) * 2,
+            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak,
+                         "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
+                         "peak_source": f"{FP4_OVER_BF16:.0f} x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s)",
+                         "traffic": None, "algorithmic_bytes": gemm_bytes,
+                         "per_shape_us": [round(t * 1e3, 2) for t in gemm_t]},
+            "rotate_quantize": {"bound": "hbm", "achieved": rq_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": rq_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                                "per_shape_us": [round(t * 1e3, 2) for t in rq_t]},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--block", type=int, default=32)
+    ap.add_argument("--ref-rows", type=int, default=0,
+                    help="rows per shape per step for --impl reference (0 = sized to finish in ~2 min)")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -33,7 +33,7 @@ def gpu_gemm(bro, ac, asc, wc, wsc, dtype, ldy=None):
     N = wc.shape[0]
     a_c, a_s = upload_operand(ac, asc)
     w_c, w_s = upload_operand(wc, wsc)
-    ldy = ldy or N
+    ldy = ldy or (N + 7) // 8 * 8          # row pitch must be a multiple of 16 bytes
     esz = 2 if dtype == torch.bfloat16 else 4
     buf = Guarded(M * ldy * esz, fill=0x7F)
     y = buf.view.view(dtype).view(M, ldy)[:, :N]
