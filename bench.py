@@ -281,10 +281,11 @@ def run_ours(args):
 
     # ---- instrumented pass: the same launches with an event after every kernel (rotate+quantize
     # and GEMM issued as the two C-ABI calls bro_linear makes), for the per-kernel roofline.
-    inst_steps = min(steps, 40)
+    inst_steps = min(steps, 24)
     rq_ms = [[] for _ in shapes]
     gemm_ms = [[] for _ in shapes]
-    for it in range(inst_steps + 3):
+    torch.cuda._sleep(int(4e7))      # hold the stream (~20 ms) while the launches below queue up,
+    for it in range(inst_steps + 3):   # so consecutive events are separated by kernel time only
         for i, (M, K, N) in enumerate(shapes):
             s = sets[i][it % ring]
             acodes = s["ws"][:bro.codes_bytes(M, K)]
@@ -348,11 +349,15 @@ def run_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        t_probe, f_probe = oracle_step(oracle_prepare(shapes, cfg, 8, block), block)
-        rows = int(max(8, min(512, 8 * 12.0 / max(t_probe, 1e-3))))
-        t, f = oracle_step(oracle_prepare(shapes, cfg, rows, block), block)
+        rows = 256
+        prepared = oracle_prepare(shapes, cfg, rows, block)
+        t, f, passes = 0.0, 0.0, 0
+        while t < 10.0 and passes < 200:          # about 10 s of CPU work
+            dt, df = oracle_step(prepared, block)
+            t, f, passes = t + dt, f + df, passes + 1
         cpu = {"value": f / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"first {rows} rows of each of the {len(shapes)} shapes, {t:.1f} s (weights packed offline, untimed)"}
+               "sample": f"first {rows} rows of each of the {len(shapes)} shapes, {passes} passes, {t:.1f} s "
+                         "(weights packed offline, untimed)"}
 
     if rank == 0:
         out = {
@@ -380,22 +385,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_rotate_quantize_only(args):
+    """Workload cfg4: the block-size sweep on a rotate+quantize-only activation tensor
+    [16384, 4096]; one step = one launch per rotation size.  Reports HBM GB/s per size
+    (2.53125 algorithmic bytes per element: 2 read, 1/2 code, 1/32 scale)."""
+    import torch
+    from paper_2511_04214_b200 import build
+    build.build()
+    from paper_2511_04214_b200 import binding as bro, synth
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    cfg = synth.CONFIGS["cfg4"]
+    M, K, _ = cfg["shapes"][0]
+    blocks = [args.block] if args.only_block else cfg["blocks"]
+    peaks = measured_peaks()
+    x0 = synth.activations(M, K, seed=cfg["seed"], recipe=cfg["recipe"]).cuda()
+    ring = 3                                                   # 3 x 128 MiB inputs > 126 MB L2
+    xs = [x0.roll(7 * r, 0).contiguous() for r in range(ring)]
+    codes = [bro.alloc_codes(M, K) for _ in range(ring)]
+    scales = [bro.alloc_scales(M, K, bro.LAYOUT_GEMM) for _ in range(ring)]
+    sampler = ClockSampler(0)
+    sampler.start()
+    per_block = {}
+    steps = args.steps
+    for _ in range(max(args.warmup, 3)):
+        for b in blocks:
+            bro.rotate_quantize_mxfp4(xs[0], b, codes[0], scales[0], bro.LAYOUT_GEMM)
+    torch.cuda.synchronize()
+    sampler.mark("t0")
+    t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(int(2e7))
+    t_all0.record()
+    evs = {b: [] for b in blocks}
+    for i in range(steps):
+        for b in blocks:
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+            c.record()
+            evs[b].append((a, c))
+    t_all1.record()
+    torch.cuda.synchronize()
+    sampler.mark("t1")
+    assert bro.last_device_status() == 0
+    bytes_per_launch = M * K * 2.53125
+    for b in blocks:
+        ts = [a.elapsed_time(c) for a, c in evs[b]]
+        per_block[str(b if b else K)] = {"us": statistics.mean(ts) * 1e3, "gbs": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9,
+                                         "frac_of_measured_copy": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    ms_total = t_all0.elapsed_time(t_all1)
+    value = bytes_per_launch * len(blocks) * steps / (ms_total * 1e-3) / 1e9
+    first = per_block[str(blocks[0] if blocks[0] else K)]
+    out = {"metric": "rotate+quantize HBM GB/s", "value": value, "unit": "GB/s", "n_gpus": 1, "steps": steps,
+           "warmup": max(args.warmup, 3), "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16 in, f32 rotation, mxfp4 out", "data": "synthetic",
+           "config": {"workload": "cfg4", "shape_MK": [M, K], "blocks": [b if b else K for b in blocks],
+                      "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm"},
+           "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
+           "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+                        "traffic": None, "algorithmic_bytes": bytes_per_launch}}
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--block", type=int, default=32)
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="rows per shape per step for --impl reference (0 = sized to finish in ~2 min)")
+    ap.add_argument("--only-block", action="store_true", help="cfg4: run only --block instead of the sweep")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "cfg4":
+        run_rotate_quantize_only(args)
     else:
         run_ours(args)
 

@@ -67,74 +67,105 @@ __device__ __forceinline__ constexpr uint32_t norm_bits() {
                           : 0x3FB504F3u - ((uint32_t)((LOG2B + 1) / 2) << 23);
 }
 
-// Quantise the 32 fp32 values v (pre-normalisation: y = v*c) of one MX group.
-// Returns the scale byte; writes 4 code words.
-__device__ __forceinline__ uint32_t quantize_group(const float (&v)[32], uint32_t cbits,
-                                                   uint32_t (&w)[4]) {
-  float m = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(v[i]));
-  const float c = __uint_as_float(cbits);
-  // amax of y: rounding is monotonic, so max_i fl(|v_i| c) = fl(max_i |v_i| * c)
-  const uint32_t ef = __float_as_uint(__fmul_rn(m, c)) >> 23;
-  const uint32_t s = ef > 2u ? ef - 2u : 0u;
-  if (ef >= 27u && ef <= 250u) {
-    // c * 2^-E is a normal fp32: one multiply, bit-identical to (v*c)*2^-E
-    const float c2 = __uint_as_float(cbits + ((127u - s) << 23));
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      w[j] = pack_e2m1x8(__fmul_rn(v[8 * j + 0], c2), __fmul_rn(v[8 * j + 1], c2),
-                         __fmul_rn(v[8 * j + 2], c2), __fmul_rn(v[8 * j + 3], c2),
-                         __fmul_rn(v[8 * j + 4], c2), __fmul_rn(v[8 * j + 5], c2),
-                         __fmul_rn(v[8 * j + 6], c2), __fmul_rn(v[8 * j + 7], c2));
-  } else {
-    const float p = __uint_as_float((254u - s) << 23);   // 2^-E, E = s - 127
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      w[j] = pack_e2m1x8(
-          __fmul_rn(__fmul_rn(v[8 * j + 0], c), p), __fmul_rn(__fmul_rn(v[8 * j + 1], c), p),
-          __fmul_rn(__fmul_rn(v[8 * j + 2], c), p), __fmul_rn(__fmul_rn(v[8 * j + 3], c), p),
-          __fmul_rn(__fmul_rn(v[8 * j + 4], c), p), __fmul_rn(__fmul_rn(v[8 * j + 5], c), p),
-          __fmul_rn(__fmul_rn(v[8 * j + 6], c), p), __fmul_rn(__fmul_rn(v[8 * j + 7], c), p));
-  }
-  return s;
+// ---- packed fp32x2 arithmetic (sm_100): one issue slot for two IEEE round-to-nearest results.
+// A group's 32 values live in 16 register pairs; pair k holds elements (2k, 2k+1).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
 
-// In-register 32-point transform, ascending stride, natural (Sylvester) order.
-__device__ __forceinline__ void fwht32(float (&v)[32]) {
+// 8 bf16 (one 16-byte chunk) -> 4 pairs, fused with butterfly stage h = 1, which pairs the two
+// halves of one 32-bit word: (lo, hi) -> (lo + hi, lo - hi).
+__device__ __forceinline__ void unpack_stage1(const uint4& q, uint64_t* P) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-  for (int h = 1; h < 32; h <<= 1) {
+  for (int k = 0; k < 4; ++k) {
+    const float lo = __uint_as_float(w[k] << 16);
+    const float hi = __uint_as_float(w[k] & 0xFFFF0000u);
+    P[k] = pack2(__fadd_rn(lo, hi), __fsub_rn(lo, hi));
+  }
+}
+
+// Butterfly stages h = 2, 4, 8, 16 on pairs (ascending stride): pair k meets pair k ^ (h/2).
+__device__ __forceinline__ void fwht32_stages_2_to_16(uint64_t (&P)[16]) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      if ((i & h) == 0) {
-        const float a = v[i], b = v[i + h];
-        v[i] = __fadd_rn(a, b);
-        v[i + h] = __fsub_rn(a, b);
+  for (int hp = 1; hp < 16; hp <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if ((k & hp) == 0) {
+        const uint64_t a = P[k], b = P[k + hp];
+        P[k] = add2(a, b);
+        P[k + hp] = sub2(a, b);
       }
     }
   }
 }
 
 // One butterfly stage across two lanes that hold the low / high half of the pairs.
-// low lane: a + b ; high lane: a - b = fma(own, -1, other) (exact, no extra rounding).
-__device__ __forceinline__ void cross_lane_stage(float (&v)[32], int lane_mask, bool is_high) {
+// low lane: a + b ; high lane: a - b = own * (-1) + other (exact, one rounding).
+__device__ __forceinline__ void cross_lane_stage(uint64_t (&P)[16], int lane_mask, bool is_high) {
   const float sgn = is_high ? -1.f : 1.f;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], lane_mask);
-    v[i] = __fmaf_rn(v[i], sgn, o);
+  for (int k = 0; k < 16; ++k) {
+    float lo, hi;
+    unpack2(P[k], lo, hi);
+    const float olo = __shfl_xor_sync(0xFFFFFFFFu, lo, lane_mask);
+    const float ohi = __shfl_xor_sync(0xFFFFFFFFu, hi, lane_mask);
+    P[k] = pack2(__fmaf_rn(lo, sgn, olo), __fmaf_rn(hi, sgn, ohi));
   }
 }
 
-__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float* v) {
-  v[0] = __uint_as_float(q.x << 16);
-  v[1] = __uint_as_float(q.x & 0xFFFF0000u);
-  v[2] = __uint_as_float(q.y << 16);
-  v[3] = __uint_as_float(q.y & 0xFFFF0000u);
-  v[4] = __uint_as_float(q.z << 16);
-  v[5] = __uint_as_float(q.z & 0xFFFF0000u);
-  v[6] = __uint_as_float(q.w << 16);
-  v[7] = __uint_as_float(q.w & 0xFFFF0000u);
+// Quantise the 32 fp32 values held in P (pre-normalisation: y = v*c) of one MX group.
+// Returns the scale byte; writes 4 code words.
+__device__ __forceinline__ uint32_t quantize_group(const uint64_t (&P)[16], uint32_t cbits, uint32_t (&w)[4]) {
+  float m = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    float lo, hi;
+    unpack2(P[k], lo, hi);
+    m = fmaxf(m, fmaxf(fabsf(lo), fabsf(hi)));
+  }
+  const float c = __uint_as_float(cbits);
+  // amax of y: rounding is monotonic, so max_i fl(|v_i| c) = fl(max_i |v_i| * c)
+  const uint32_t ef = __float_as_uint(__fmul_rn(m, c)) >> 23;
+  const uint32_t s = ef > 2u ? ef - 2u : 0u;
+  float r[32];
+  if (ef >= 27u && ef <= 250u) {
+    // c * 2^-E is a normal fp32: one multiply, bit-identical to (v*c)*2^-E
+    const float c2 = __uint_as_float(cbits + ((127u - s) << 23));
+    const uint64_t cc = pack2(c2, c2);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) unpack2(mul2(P[k], cc), r[2 * k], r[2 * k + 1]);
+  } else {
+    const float p2 = __uint_as_float((254u - s) << 23);   // 2^-E, E = s - 127
+    const uint64_t cc = pack2(c, c), pp = pack2(p2, p2);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) unpack2(mul2(mul2(P[k], cc), pp), r[2 * k], r[2 * k + 1]);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    w[j] = pack_e2m1x8(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3], r[8 * j + 4], r[8 * j + 5],
+                       r[8 * j + 6], r[8 * j + 7]);
+  return s;
 }
 
 template <int LOG2B>
@@ -167,19 +198,23 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
       uint32_t phase = 0;
       bool ok = true;
       int64_t issued = 0;
+      const int tiles_k = (int)p.tiles_k;
+      int tm = (int)(blockIdx.x / (unsigned)tiles_k), tk = (int)(blockIdx.x % (unsigned)tiles_k);
+      const int step_m = (int)(gridDim.x / (unsigned)tiles_k), step_k = (int)(gridDim.x % (unsigned)tiles_k);
       for (int64_t t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-        const int64_t tm = t / p.tiles_k, tk = t - tm * p.tiles_k;
         if (issued >= kStages)
           ok = mbar_wait(bar_base + 8 * (kStages + stage), phase ^ 1u, SITE_RQ_EMPTY);
         if (!ok) break;
         const uint32_t full = bar_base + 8 * stage;
         const uint32_t dst = smem_base + stage * kStageBytes;
         mbar_arrive_expect_tx(full, kStageBytes);
-        tma_load_2d(dst, &tmx, (int)(tk * kTileCols), (int)(tm * kTileRows), full);
-        tma_load_2d(dst + kBoxBytes, &tmx, (int)(tk * kTileCols + kBoxCols),
-                    (int)(tm * kTileRows), full);
+        tma_load_2d(dst, &tmx, tk * kTileCols, tm * kTileRows, full);
+        tma_load_2d(dst + kBoxBytes, &tmx, tk * kTileCols + kBoxCols, tm * kTileRows, full);
         ++issued;
         if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        tm += step_m;
+        tk += step_k;
+        if (tk >= tiles_k) { tk -= tiles_k; ++tm; }
       }
       if (!ok) {
         // A consumer gave up.  Do not leave the CTA while copies may still land in its shared
@@ -203,30 +238,32 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
 
     int stage = 0;
     uint32_t phase = 0;
+    const int tiles_k = (int)p.tiles_k;
+    int tm = (int)(blockIdx.x / (unsigned)tiles_k), tk = (int)(blockIdx.x % (unsigned)tiles_k);
+    const int step_m = (int)(gridDim.x / (unsigned)tiles_k), step_k = (int)(gridDim.x % (unsigned)tiles_k);
     for (int64_t t = blockIdx.x; t < total_tiles; t += gridDim.x) {
-      const int64_t tm = t / p.tiles_k, tk = t - tm * p.tiles_k;
       if (!mbar_wait(bar_base + 8 * stage, phase, SITE_RQ_FULL)) break;
       const uint32_t src = smem_base + stage * kStageBytes + row_off;
-      float v[32];
+      uint64_t P[16];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint4 q = lds128(src + ((((uint32_t)gg * 4u + j) ^ sw) << 4));
-        unpack_bf16x8(q, v + 8 * j);
+        unpack_stage1(q, P + 4 * j);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_base + 8 * (kStages + stage));
       if (++stage == kStages) { stage = 0; phase ^= 1u; }
 
-      fwht32(v);
-      if (LOG2B >= 6) cross_lane_stage(v, 1, gg != 0);
-      if (LOG2B >= 7) cross_lane_stage(v, 8, box != 0);
+      fwht32_stages_2_to_16(P);
+      if (LOG2B >= 6) cross_lane_stage(P, 1, gg != 0);
+      if (LOG2B >= 7) cross_lane_stage(P, 8, box != 0);
 
       uint32_t w[4];
-      const uint32_t s = quantize_group(v, cbits, w);
+      const uint32_t s = quantize_group(P, cbits, w);
 
-      const int64_t grow = tm * kTileRows + row;
-      const int64_t ggrp = tk * (kTileCols / 32) + g;     // group index along K
-      const bool in_k = ggrp * 32 < p.K;
+      const int64_t grow = (int64_t)tm * kTileRows + row;
+      const int ggrp = tk * (kTileCols / 32) + g;         // group index along K
+      const bool in_k = ggrp * 32 < (int)p.K;
       if (grow < p.M && in_k) {
         uint4* dst = reinterpret_cast<uint4*>(p.codes + grow * (p.K >> 1) + ggrp * 16);
         *dst = make_uint4(w[0], w[1], w[2], w[3]);
@@ -238,10 +275,10 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
       if (g == 0) {
         if (p.layout == BRO_LAYOUT_GEMM) {
           // 512-byte block (tm, tk): byte (r%32)*16 + (r/32)*4 + g ; padding rows included
-          const int64_t off = (tm * p.scale_kblocks + tk) * 512 + (row & 31) * 16 + (row >> 5) * 4;
+          const int64_t off = ((int64_t)tm * p.scale_kblocks + tk) * 512 + (row & 31) * 16 + (row >> 5) * 4;
           *reinterpret_cast<uint32_t*>(p.scales + off) = sb;
         } else if (grow < p.M) {
-          const int64_t ng = p.K >> 5;
+          const int ng = (int)(p.K >> 5);
           uint8_t* dst = p.scales + grow * ng + tk * 4;
           if (tk * 4 + 4 <= ng && ((reinterpret_cast<uintptr_t>(dst) & 3) == 0)) {
             *reinterpret_cast<uint32_t*>(dst) = sb;
@@ -250,6 +287,9 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
           }
         }
       }
+      tm += step_m;
+      tk += step_k;
+      if (tk >= tiles_k) { tk -= tiles_k; ++tm; }
     }
   }
 }

@@ -41,32 +41,32 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   for (int64_t it = blockIdx.x; it < row_iters; it += gridDim.x) {
     const int64_t row = it * p.rows_per_iter + rs;
     const bool live = row < p.M;
-    float v[32];
-    if (live) {
-      const uint4* src = reinterpret_cast<const uint4*>(p.x + row * p.ldx + (int64_t)gi * 32);
+    uint64_t P[16];
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(p.x + (live ? row : 0) * p.ldx + (int64_t)gi * 32);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint4 q = __ldg(src + j);
-        rq::unpack_bf16x8(q, v + 8 * j);
+        const uint4 q = live ? __ldg(src + j) : make_uint4(0u, 0u, 0u, 0u);
+        rq::unpack_stage1(q, P + 4 * j);
       }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = 0.f;
     }
-    rq::fwht32(v);
+    rq::fwht32_stages_2_to_16(P);
     // lane stages: stride 32 * m, m = 1..16 (only those below K)
 #pragma unroll
     for (int m = 1; m < 32; m <<= 1) {
-      if (m < T) rq::cross_lane_stage(v, m, (gi & m) != 0);
+      if (m < T) rq::cross_lane_stage(P, m, (gi & m) != 0);
     }
     // warp stages through shared memory
     for (int m = 32; m < T; m <<= 1) {
       float* mine = xch + (size_t)rs * p.K + (size_t)gi * 32;
       __syncthreads();   // previous round's reads are done
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<float4*>(mine + ((c ^ (gi & 7)) << 2)) =
-            make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+      for (int c = 0; c < 8; ++c) {
+        float a0, a1, a2, a3;
+        rq::unpack2(P[2 * c], a0, a1);
+        rq::unpack2(P[2 * c + 1], a2, a3);
+        *reinterpret_cast<float4*>(mine + ((c ^ (gi & 7)) << 2)) = make_float4(a0, a1, a2, a3);
+      }
       __syncthreads();
       const int pg = gi ^ m;
       const float* theirs = xch + (size_t)rs * p.K + (size_t)pg * 32;
@@ -74,14 +74,15 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const float4 o = *reinterpret_cast<const float4*>(theirs + ((c ^ (pg & 7)) << 2));
-        v[4 * c + 0] = __fmaf_rn(v[4 * c + 0], sgn, o.x);
-        v[4 * c + 1] = __fmaf_rn(v[4 * c + 1], sgn, o.y);
-        v[4 * c + 2] = __fmaf_rn(v[4 * c + 2], sgn, o.z);
-        v[4 * c + 3] = __fmaf_rn(v[4 * c + 3], sgn, o.w);
+        float a0, a1, a2, a3;
+        rq::unpack2(P[2 * c], a0, a1);
+        rq::unpack2(P[2 * c + 1], a2, a3);
+        P[2 * c] = rq::pack2(__fmaf_rn(a0, sgn, o.x), __fmaf_rn(a1, sgn, o.y));
+        P[2 * c + 1] = rq::pack2(__fmaf_rn(a2, sgn, o.z), __fmaf_rn(a3, sgn, o.w));
       }
     }
     uint32_t w[4];
-    const uint32_t s = rq::quantize_group(v, cbits, w);
+    const uint32_t s = rq::quantize_group(P, cbits, w);
     if (live) {
       *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (int64_t)gi * 16) =
           make_uint4(w[0], w[1], w[2], w[3]);
