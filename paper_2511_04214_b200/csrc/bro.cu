@@ -105,6 +105,12 @@ bro_status bro::gemm::make_codes_map(CUtensorMap* map, const void* base, int64_t
                      (uint64_t)(K / 2), 128, (uint32_t)box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// bf16 output [M, ldy]: box = 32 columns (64 bytes) x 128 rows, 64-byte swizzle (epilogue staging).
+bro_status bro::gemm::make_out_map(CUtensorMap* map, const void* y, int64_t M, int64_t N, int64_t ldy) {
+  return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy * 2,
+                     bro::gemm::kChunkCols, bro::gemm::kBM, CU_TENSOR_MAP_SWIZZLE_64B);
+}
+
 namespace {
 
 // ---- rotate + quantise ---------------------------------------------------------------------------

@@ -3,18 +3,27 @@
 //
 //   y[m, n] = sum_g 2^(Ea[m,g] + Ew[n,g]) * sum_{k in g} a[m,k] w[n,k]
 //
-// One CTA computes a 128 x BN output tile.  Warp-specialised:
+// Persistent kernel, one CTA per SM, 128 x BN output tiles handed out round-robin.
+// Warp-specialised, every role loops over the CTA's tiles so that the stages of consecutive
+// tiles overlap:
 //   warp 0      TMA producer: per 256-element K step, one 128x128-byte box of A codes, one
 //               BNx128-byte box of W codes (128-byte swizzle) and the matching 512-byte scale
 //               blocks (plain bulk copies; the scale tensors are already in tensor-core order).
+//               The shared-memory ring runs ahead across tile boundaries.
 //   warp 1      owns TMEM; one elected thread copies the scale blocks shared -> TMEM
 //               (tcgen05.cp) and issues four tcgen05.mma kind::mxf4.block_scale (K = 64 each)
-//               per K step into a 128 x BN fp32 accumulator in TMEM; tcgen05.commit releases the
-//               shared-memory stage and finally signals the epilogue.
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (one TMEM lane quadrant per warp), convert,
-//               store.
+//               per K step into one of two fp32 accumulators in TMEM; tcgen05.commit releases the
+//               shared-memory stage and, after the last K step, hands the accumulator over.
+//   warps 2..5  epilogue: tcgen05.ld the accumulator in 32-column chunks (one TMEM lane quadrant
+//               per warp), convert to bf16, stage the chunk in shared memory (64-byte swizzle)
+//               and write it with a TMA store (which also clips the ragged edges); the fp32
+//               output mode stores straight from registers.
+// TMEM holds 512 columns.  For BN = 256 two full accumulators plus the scale columns do not
+// fit, so the two accumulators overlap by 32 columns ([0,256) and [224,480)): the epilogue drains
+// the shared 32 columns first and releases them early, and the next tile's MMAs start as soon as
+// those columns and the rest of its own buffer are free.
 // Every mbarrier wait is bounded; on expiry the role records the site and falls through to the
-// common exit, where TMEM is released.
+// common exit, where outstanding copies are awaited and TMEM is released.
 #pragma once
 
 #include <stdlib.h>
@@ -28,17 +37,22 @@ constexpr int kBM = 128;
 constexpr int kBK = 256;                    // elements per K step = 128 bytes of codes per row
 constexpr int kThreads = 192;
 constexpr int kATileBytes = kBM * 128;      // 16 KiB
+constexpr int kChunkCols = 32;              // epilogue chunk: 32 fp32 columns per tcgen05.ld
+constexpr int kStageOutBytes = kBM * kChunkCols * 2;   // 8 KiB bf16 staging per chunk
 
 template <int BN> struct Cfg {
-  static constexpr int kStages = BN == 256 ? 4 : 3;
+  static constexpr int kStages = BN == 256 ? 4 : 6;
   static constexpr int kBTileBytes = BN * 128;
   static constexpr int kSfaBytes = 1024;                  // 2 blocks of 512 B (128 rows x 4 groups)
   static constexpr int kSfbBytes = (BN / 128) * 1024;
   static constexpr int kStageBytes = kATileBytes + kBTileBytes + kSfaBytes + kSfbBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
-  static constexpr int kSfaCols = 8;                      // 2 K-blocks x 4 columns
-  static constexpr int kSfbCols = (BN / 32) * 2;          // 2 K-blocks x BN/32 columns
-  static constexpr int kTmemCols = BN == 256 ? 512 : 256; // power of two >= BN + SF columns
+  static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kStageOutBytes + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int kTmemCols = 512;
+  static constexpr int kAccStride = BN == 256 ? 224 : BN;   // column offset of accumulator 1
+  static constexpr bool kOverlap = BN == 256;               // accumulators share 32 columns
+  static constexpr int kSfaCol = 480;                       // 8 columns: 2 K-blocks x 4
+  static constexpr int kSfbCol = 488;                       // up to 16 columns: 2 K-blocks x BN/32
+  static constexpr int kChunks = BN / kChunkCols;
 };
 
 struct Params {
@@ -48,6 +62,7 @@ struct Params {
   int64_t M, N, K, ldy;
   int64_t kblocks;          // 512-byte scale blocks per 128-row block = 2*ceil(K/256)
   int num_k_steps;          // ceil(K/256)
+  int tiles_m, tiles_n, total_tiles;
 };
 
 // ---- tcgen05 wrappers ------------------------------------------------------------------------
@@ -118,9 +133,42 @@ __device__ __forceinline__ constexpr uint32_t make_idesc() {
          ((uint32_t)(kBM >> 4) << 24);
 }
 
+
+// Barrier over `nthreads` threads that also ANDs a predicate, so that all of them take the same
+// branch afterwards (used to leave the tile loop together after a lost wait).
+__device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{ .reg .pred p, q; setp.ne.u32 q, %3, 0; bar.red.and.pred p, %1, %2, q; selp.u32 %0, 1, 0, p; }"
+      : "=r"(out)
+      : "r"(id), "r"(nthreads), "r"((uint32_t)pred)
+      : "memory");
+  return out != 0;
+}
+__device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// TMA store shared -> global of one box; out-of-range parts of the box are clipped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(m)),
+               "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 template <int BN, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw, const Params p) {
+gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw,
+                  const __grid_constant__ CUtensorMap tmy, const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -128,26 +176,29 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   const uint32_t sB = sA + C::kStages * kATileBytes;
   const uint32_t sSFA = sB + C::kStages * C::kBTileBytes;
   const uint32_t sSFB = sSFA + C::kStages * C::kSfaBytes;
-  const uint32_t bar_base = sSFB + C::kStages * C::kSfbBytes;
-  const uint32_t bar_full = bar_base;                       // [kStages]
-  const uint32_t bar_empty = bar_base + 8 * C::kStages;     // [kStages]
-  const uint32_t bar_acc = bar_base + 16 * C::kStages;      // accumulator ready
-  const uint32_t tmem_slot = bar_acc + 8;                   // u32 written by tcgen05.alloc
-  uint32_t* tmem_slot_ptr =
-      reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+  const uint32_t sOut = sSFB + C::kStages * C::kSfbBytes;          // 2 x 8 KiB, 1 KiB aligned
+  const uint32_t bar_base = sOut + 2 * kStageOutBytes;
+  const uint32_t bar_full = bar_base;                              // [kStages]
+  const uint32_t bar_empty = bar_base + 8 * C::kStages;            // [kStages]
+  const uint32_t bar_acc_full = bar_base + 16 * C::kStages;        // [2] MMA -> epilogue
+  const uint32_t bar_acc_free = bar_acc_full + 16;                 // [2] epilogue -> MMA, whole buffer
+  const uint32_t bar_ovl_free = bar_acc_free + 16;                 // [2] epilogue -> MMA, shared columns
+  const uint32_t tmem_slot = bar_ovl_free + 16;                    // u32 written by tcgen05.alloc
+  uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int64_t m0 = (int64_t)blockIdx.y * kBM;
-  const int64_t n0 = (int64_t)blockIdx.x * BN;
-  const int nblk_valid = (n0 + 128 < p.N && BN == 256) ? 2 : 1;   // 128-row scale blocks of W in range
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
-    mbar_init(bar_acc, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_acc_full + 8 * b, 1);
+      mbar_init(bar_acc_free + 8 * b, 4);    // one arrival per epilogue warp
+      mbar_init(bar_ovl_free + 8 * b, 4);
+    }
     mbar_fence_init();
     fence_proxy_async_smem();
   }
@@ -159,9 +210,8 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-  const uint32_t tmem_acc = tmem_base;
-  const uint32_t tmem_sfa = tmem_base + BN;
-  const uint32_t tmem_sfb = tmem_base + BN + C::kSfaCols;
+  const uint32_t tmem_sfa = tmem_base + C::kSfaCol;
+  const uint32_t tmem_sfb = tmem_base + C::kSfbCol;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -170,28 +220,33 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
       tma_prefetch_desc(&tmw);
       int stage = 0;
       uint32_t phase = 0;
-      int issued = 0;
+      int64_t issued = 0;
       bool ok = true;
-      const uint8_t* sfa_src = p.ascales + (int64_t)blockIdx.y * p.kblocks * 512;
-      const uint8_t* sfb_src = p.wscales + (n0 / 128) * p.kblocks * 512;
-      for (int ks = 0; ks < p.num_k_steps; ++ks) {
-        if (issued >= C::kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
-        if (!ok) break;
-        const uint32_t full = bar_full + 8 * stage;
-        mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
-        tma_load_2d(sA + stage * kATileBytes, &tma, ks * 128, (int)m0, full);
-        tma_load_2d(sB + stage * C::kBTileBytes, &tmw, ks * 128, (int)n0, full);
-        bulk_load_1d(sSFA + stage * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
-        for (int nb = 0; nb < nblk_valid; ++nb)
-          bulk_load_1d(sSFB + stage * C::kSfbBytes + nb * 1024,
-                       sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512, 1024, full);
-        ++issued;
-        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+        const int m0 = tm * kBM, n0 = tn * BN;
+        const int nblk_valid = (BN == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1;
+        const uint8_t* sfa_src = p.ascales + (int64_t)tm * p.kblocks * 512;
+        const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
+        for (int ks = 0; ks < p.num_k_steps; ++ks) {
+          if (issued >= C::kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
+          if (!ok) break;
+          const uint32_t full = bar_full + 8 * stage;
+          mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
+          tma_load_2d(sA + stage * kATileBytes, &tma, ks * 128, m0, full);
+          tma_load_2d(sB + stage * C::kBTileBytes, &tmw, ks * 128, n0, full);
+          bulk_load_1d(sSFA + stage * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
+          for (int nb = 0; nb < nblk_valid; ++nb)
+            bulk_load_1d(sSFB + stage * C::kSfbBytes + nb * 1024,
+                         sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512, 1024, full);
+          ++issued;
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
       }
       if (!ok) {
-        const int first = issued > C::kStages ? issued - C::kStages : 0;
-        for (int i = first; i < issued; ++i)
-          mbar_wait(bar_full + 8 * (i % C::kStages), (uint32_t)((i / C::kStages) & 1), SITE_GEMM_DRAIN);
+        const int64_t first = issued > C::kStages ? issued - C::kStages : 0;
+        for (int64_t i = first; i < issued; ++i)
+          mbar_wait(bar_full + 8 * (int)(i % C::kStages), (uint32_t)((i / C::kStages) & 1), SITE_GEMM_DRAIN);
       }
     }
   } else if (warp == 1) {
@@ -201,76 +256,126 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int ks = 0; ks < p.num_k_steps && ok; ++ks) {
-        ok = mbar_wait(bar_full + 8 * stage, phase, SITE_GEMM_FULL);
+      int it = 0;   // index of this CTA's tile
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const int use = it >> 1;                       // how many times this buffer was used before
+        // this buffer must have been drained by the epilogue of tile it-2 ...
+        if (use >= 1) ok = mbar_wait(bar_acc_free + 8 * buf, (uint32_t)((use - 1) & 1), SITE_GEMM_ACC_EMPTY);
+        // ... and the columns it shares with the other buffer by the epilogue of tile it-1
+        if (ok && C::kOverlap && it >= 1)
+          ok = mbar_wait(bar_ovl_free + 8 * (buf ^ 1), (uint32_t)(((it - 1) >> 1) & 1), SITE_GEMM_ACC_EMPTY);
         if (!ok) break;
         tc_fence_after();
-        // scale blocks of this K step: shared -> TMEM.  K-block pair a (128 elements) of A goes to
-        // columns 4a..4a+3; of W to columns (BN/32)*a + 4*nb .. +3.
+        const uint32_t tmem_acc = tmem_base + buf * C::kAccStride;
+        for (int ks = 0; ks < p.num_k_steps; ++ks) {
+          ok = mbar_wait(bar_full + 8 * stage, phase, SITE_GEMM_FULL);
+          if (!ok) break;
+          tc_fence_after();
+          // scale blocks of this K step: shared -> TMEM.  K-block pair a (128 elements) of A goes to
+          // columns 4a..4a+3; of W to columns (BN/32)*a + 4*nb .. +3.
 #pragma unroll
-        for (int a = 0; a < 2; ++a) {
-          tc_cp_sf(tmem_sfa + 4 * a, smem_desc_sf(sSFA + stage * C::kSfaBytes + a * 512));
+          for (int a = 0; a < 2; ++a) {
+            tc_cp_sf(tmem_sfa + 4 * a, smem_desc_sf(sSFA + stage * C::kSfaBytes + a * 512));
 #pragma unroll
-          for (int nb = 0; nb < BN / 128; ++nb)
-            tc_cp_sf(tmem_sfb + (BN / 32) * a + 4 * nb,
-                     smem_desc_sf(sSFB + stage * C::kSfbBytes + nb * 1024 + a * 512));
+            for (int nb = 0; nb < BN / 128; ++nb)
+              tc_cp_sf(tmem_sfb + (BN / 32) * a + 4 * nb,
+                       smem_desc_sf(sSFB + stage * C::kSfbBytes + nb * 1024 + a * 512));
+          }
+          const uint64_t adesc = smem_desc_sw128(sA + stage * kATileBytes);
+          const uint64_t bdesc = smem_desc_sw128(sB + stage * C::kBTileBytes);
+#pragma unroll
+          for (int kb = 0; kb < 4; ++kb) {
+            const uint32_t sf_id = (kb & 1) * 2;          // bytes {0,1} or {2,3} of the scale word
+            const uint32_t idesc = idesc0 | (sf_id << 4) | (sf_id << 29);
+            const uint32_t tsfa = (tmem_sfa + 4 * (kb >> 1)) | (sf_id << 30);
+            const uint32_t tsfb = (tmem_sfb + (BN / 32) * (kb >> 1)) | (sf_id << 30);
+            tc_mma_mxf4(tmem_acc, adesc + 2 * kb, bdesc + 2 * kb, idesc, tsfa, tsfb, (ks | kb) != 0 ? 1u : 0u);
+          }
+          tc_commit(bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
-        const uint64_t adesc = smem_desc_sw128(sA + stage * kATileBytes);
-        const uint64_t bdesc = smem_desc_sw128(sB + stage * C::kBTileBytes);
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          const uint32_t sf_id = (kb & 1) * 2;            // bytes {0,1} or {2,3} of the scale word
-          const uint32_t idesc = idesc0 | (sf_id << 4) | (sf_id << 29);
-          const uint32_t tsfa = (tmem_sfa + 4 * (kb >> 1)) | (sf_id << 30);
-          const uint32_t tsfb = (tmem_sfb + (BN / 32) * (kb >> 1)) | (sf_id << 30);
-          tc_mma_mxf4(tmem_acc, adesc + 2 * kb, bdesc + 2 * kb, idesc, tsfa, tsfb, (ks | kb) != 0 ? 1u : 0u);
-        }
-        tc_commit(bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
-        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        tc_commit(bar_acc_full + 8 * buf);    // accumulator complete (or abandoned) -> epilogue
       }
-      tc_commit(bar_acc);                   // accumulator complete (or abandoned) -> epilogue
     }
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
-    const bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc, 0, SITE_GEMM_ACC_FULL));
-    tc_fence_after();
-    const int64_t row = m0 + q * 32 + lane;
-    if (ok) {
+    const int ep_tid = threadIdx.x - 64;    // 0..127
+    const int r_in_tile = q * 32 + lane;
+    uint32_t chunk_counter = 0;             // staging buffer = chunk_counter & 1
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++it) {
+      const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+      const int m0 = tm * kBM, n0 = tn * BN;
+      const int buf = it & 1;
+      ok = named_barrier_and(2, 128, mbar_wait(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tmem_acc = tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16);
+      const int64_t row = (int64_t)m0 + r_in_tile;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int ci = 0; ci < C::kChunks; ++ci) {
+        // Chunk order: the columns shared with the other accumulator first.  Buffer 0 shares its
+        // last chunk, buffer 1 its first.
+        const int c = (C::kOverlap && buf == 0) ? (ci == 0 ? C::kChunks - 1 : ci - 1) : ci;
         uint32_t r[32];
-        tc_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
+        tc_ld32(tmem_acc + c * kChunkCols, r);
         tc_wait_ld();
-        const int64_t col0 = n0 + c * 32;
-        if (row < p.M && col0 < p.N) {
-          if (OUT_F32) {
+        if (ci == 0 || ci == C::kChunks - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (ci == 0) mbar_arrive(bar_ovl_free + 8 * buf);
+            if (ci == C::kChunks - 1) mbar_arrive(bar_acc_free + 8 * buf);
+          }
+        }
+        const int col0 = n0 + c * kChunkCols;
+        if (OUT_F32) {
+          if (row < p.M && col0 < p.N) {
             float* dst = static_cast<float*>(p.y) + row * p.ldy + col0;
-            if (col0 + 32 <= p.N) {
+            if ((int64_t)col0 + 32 <= p.N) {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
                 reinterpret_cast<uint4*>(dst)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
             } else {
               for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __uint_as_float(r[j]);
             }
-          } else {
-            uint16_t* dst = static_cast<uint16_t*>(p.y) + row * p.ldy + col0;
-            uint32_t h[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r[2 * j + 1])), "f"(__uint_as_float(r[2 * j])));
-            if (col0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-                reinterpret_cast<uint4*>(dst)[j] = make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-            } else {
-              for (int j = 0; j < 32 && col0 + j < p.N; ++j)
-                dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFF));
-            }
           }
+        } else {
+          uint32_t h[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r[2 * j + 1])), "f"(__uint_as_float(r[2 * j])));
+          const uint32_t sbuf = sOut + (chunk_counter & 1u) * kStageOutBytes;
+          // the TMA store that last read this staging buffer (two chunks ago) must be done reading
+          if (ep_tid == 0) bulk_wait_read<1>();
+          named_barrier_sync(1, 128);
+          // row r of the chunk: 64 bytes at r*64, 16-byte pieces XOR-swizzled with (r >> 1) & 3
+          const uint32_t rowaddr = sbuf + (uint32_t)r_in_tile * 64u;
+          const uint32_t sw = ((uint32_t)r_in_tile >> 1) & 3u;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            sts128(rowaddr + ((j ^ sw) << 4), h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+          fence_proxy_async_smem();
+          named_barrier_sync(1, 128);
+          // A TMA store clips at 16-byte granularity: when N is not a multiple of 8 the ragged last
+          // chunk is written from registers instead, element by element.
+          const bool ragged = ((p.N & 7) != 0) && ((int64_t)col0 + kChunkCols > p.N);
+          if (ep_tid == 0 && col0 < p.N && !ragged) tma_store_2d(&tmy, sbuf, col0, m0);
+          if (ep_tid == 0) bulk_commit();     // (possibly empty) keeps the group count in step
+          if (ragged && row < p.M) {
+            uint16_t* dst = static_cast<uint16_t*>(p.y) + row * p.ldy + col0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if ((int64_t)col0 + j < p.N) dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
+          }
+          ++chunk_counter;
         }
       }
     }
+    if (!OUT_F32 && ep_tid == 0) bulk_wait_all();
   }
   tc_fence_before();
   __syncthreads();
@@ -280,13 +385,19 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
 inline size_t workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 
 bro_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int box_rows);
+bro_status make_out_map(CUtensorMap* map, const void* y, int64_t M, int64_t N, int64_t ldy);
 
 template <int BN>
-bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const Params& p, int out_dtype,
-                       cudaStream_t st) {
+bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUtensorMap& tmy, Params& p,
+                       int out_dtype, int sm_count, cudaStream_t st) {
   using C = Cfg<BN>;
-  dim3 grid((unsigned)((p.N + BN - 1) / BN), (unsigned)((p.M + kBM - 1) / kBM));
-  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
+  p.tiles_m = (int)((p.M + kBM - 1) / kBM);
+  p.tiles_n = (int)((p.N + BN - 1) / BN);
+  const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
+  if (total > 0x7FFFFFFF) return BRO_ERR_UNSUPPORTED;
+  p.total_tiles = (int)total;
+  const int grid = (int)(total < sm_count ? total : sm_count);
+  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
     static bool attr_done[64][2] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -296,7 +407,7 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const Par
         return BRO_ERR_CUDA;
       attr_done[dev][which] = true;
     }
-    kernel<<<grid, kThreads, C::kSmemBytes, st>>>(tma, tmw, p);
+    kernel<<<grid, kThreads, C::kSmemBytes, st>>>(tma, tmw, tmy, p);
     return cuda_ok(cudaGetLastError(), "gemm_mxfp4 launch") ? BRO_OK : BRO_ERR_CUDA;
   };
   return out_dtype == BRO_OUT_F32 ? go(gemm_mxfp4_kernel<BN, true>, 1) : go(gemm_mxfp4_kernel<BN, false>, 0);
@@ -304,8 +415,7 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const Par
 
 inline bro_status launch(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
                          int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* /*ws*/,
-                         size_t /*ws_bytes*/, int /*sm_count*/, cudaStream_t st) {
-  if ((M + kBM - 1) / kBM > 65535) return BRO_ERR_UNSUPPORTED;
+                         size_t /*ws_bytes*/, int sm_count, cudaStream_t st) {
   int bn = 256;
   if (const char* e = getenv("BRO_GEMM_TILE_N")) bn = atoi(e) == 128 ? 128 : 256;
   else if (N <= 128) bn = 128;
@@ -316,12 +426,19 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   p.M = M; p.N = N; p.K = K; p.ldy = ldy;
   p.num_k_steps = (int)((K + kBK - 1) / kBK);
   p.kblocks = 2 * (int64_t)p.num_k_steps;
-  CUtensorMap tma, tmw;
+  CUtensorMap tma, tmw, tmy;
   bro_status rc = make_codes_map(&tma, acodes, M, K, kBM);
   if (rc != BRO_OK) return rc;
   rc = make_codes_map(&tmw, wcodes, N, K, bn);
   if (rc != BRO_OK) return rc;
-  return bn == 256 ? launch_tile<256>(tma, tmw, p, out_dtype, st) : launch_tile<128>(tma, tmw, p, out_dtype, st);
+  if (out_dtype == BRO_OUT_BF16) {
+    rc = make_out_map(&tmy, y, M, N, ldy);
+    if (rc != BRO_OK) return rc;
+  } else {
+    tmy = tma;   // unused by the fp32-output kernel
+  }
+  return bn == 256 ? launch_tile<256>(tma, tmw, tmy, p, out_dtype, sm_count, st)
+                   : launch_tile<128>(tma, tmw, tmy, p, out_dtype, sm_count, st);
 }
 
 }  // namespace gemm
