@@ -40,6 +40,15 @@ def workload_shapes(name):
     return cfg, shapes
 
 
+def select_shapes(args):
+    """The workload's shapes, or the single one picked with --shape-index (seed offsets kept)."""
+    cfg, shapes = workload_shapes(args.workload)
+    idx = list(range(len(shapes)))
+    if args.shape_index >= 0:
+        idx = [args.shape_index]
+    return cfg, [shapes[i] for i in idx], idx
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -113,13 +122,14 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-def oracle_prepare(shapes, cfg, rows_per_shape, block):
+def oracle_prepare(shapes, cfg, rows_per_shape, block, idx=None):
     """Inputs for the CPU oracle: the first `rows_per_shape` rows of every shape, weights packed by
     the oracle (offline, untimed)."""
     import oracle
     from paper_2511_04214_b200 import synth
     prepared = []
-    for i, (M, K, N) in enumerate(shapes):
+    for j, (M, K, N) in enumerate(shapes):
+        i = idx[j] if idx is not None else j
         m = min(M, rows_per_shape)
         x = synth.activations(m, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
         w = synth.weights(N, K, seed=cfg["seed"] + i)
@@ -146,13 +156,13 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    cfg, shapes = workload_shapes(args.workload)
+    cfg, shapes, idx = select_shapes(args)
     rows = args.ref_rows
     if rows <= 0:
-        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block), args.block)
-        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block), args.block)
+        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block, idx), args.block)
+        t1, _ = oracle_step(oracle_prepare(shapes, cfg, 1, args.block, idx), args.block)
         rows = int(max(1, min(64, 120.0 / (max(args.steps + args.warmup, 1) * max(t1, 1e-4)))))
-    prepared = oracle_prepare(shapes, cfg, rows, args.block)
+    prepared = oracle_prepare(shapes, cfg, rows, args.block, idx)
     for _ in range(max(args.warmup, 0)):
         oracle_step(prepared, args.block)
     total_t, total_f = 0.0, 0.0
@@ -195,7 +205,7 @@ def run_ours(args):
         dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist = dist_mod
     dev = torch.device("cuda", local_rank)
-    cfg, shapes = workload_shapes(args.workload)
+    cfg, shapes, idx = select_shapes(args)
     block = args.block
     peaks = measured_peaks()
 
@@ -205,7 +215,8 @@ def run_ours(args):
     ring = max(2, min(8, -(-3 * L2_BYTES // per_step_bytes)))
     sets = []
     stream = torch.cuda.current_stream()
-    for i, (M, K, N) in enumerate(shapes):
+    for j, (M, K, N) in enumerate(shapes):
+        i = idx[j]
         w = synth.weights(N, K, seed=cfg["seed"] + i).to(dev)
         x0 = synth.activations(M, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
         ws_bytes = bro.linear_workspace_bytes(M, N, K)
@@ -279,30 +290,41 @@ def run_ours(args):
         raise SystemExit(f"device status {bro.status_string(status)} after the timed region")
     value = flops_per_step * steps * world / (ms_total * 1e-3) / 1e12
 
-    # ---- instrumented pass: the same launches with an event after every kernel (rotate+quantize
-    # and GEMM issued as the two C-ABI calls bro_linear makes), for the per-kernel roofline.
-    inst_steps = min(steps, 24)
+    # ---- instrumented pass for the per-kernel roofline: the two C-ABI calls bro_linear makes,
+    # each timed with CUDA events around a group of `ring` back-to-back launches (one per ring
+    # set, so no launch finds its operands in L2); per-launch time = group time / ring.  Timing
+    # every launch with its own pair of events adds microseconds of event latency to kernels
+    # that only run for ten.
+    inst_steps = max(3, min(steps // ring, 16))
     rq_ms = [[] for _ in shapes]
     gemm_ms = [[] for _ in shapes]
-    torch.cuda._sleep(int(4e7))      # hold the stream (~20 ms) while the launches below queue up,
-    for it in range(inst_steps + 3):   # so consecutive events are separated by kernel time only
+
+    def views(i, r):
+        M, K, N = shapes[i]
+        s = sets[i][r]
+        nc = bro.codes_bytes(M, K)
+        off = (nc + 1023) // 1024 * 1024
+        return s, s["ws"][:nc], s["ws"][off:off + bro.scales_bytes(M, K, bro.LAYOUT_GEMM)]
+
+    torch.cuda._sleep(int(4e7))        # hold the stream (~20 ms) while the launches below queue up
+    for it in range(inst_steps + 2):
         for i, (M, K, N) in enumerate(shapes):
-            s = sets[i][it % ring]
-            acodes = s["ws"][:bro.codes_bytes(M, K)]
-            off = (bro.codes_bytes(M, K) + 1023) // 1024 * 1024
-            ascales = s["ws"][off:off + bro.scales_bytes(M, K, bro.LAYOUT_GEMM)]
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
             ev[0].record()
-            bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
+            for r in range(ring):
+                s, acodes, ascales = views(i, r)
+                bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
             ev[1].record()
-            bro.gemm_mxfp4(acodes, ascales, s["wcodes"], s["wscales"], M, N, K, s["y"])
+            for r in range(ring):
+                s, acodes, ascales = views(i, r)
+                bro.gemm_mxfp4(acodes, ascales, s["wcodes"], s["wscales"], M, N, K, s["y"])
             ev[2].record()
-            if it >= 3:
+            if it >= 2:
                 rq_ms[i].append((ev[0], ev[1]))
                 gemm_ms[i].append((ev[1], ev[2]))
     torch.cuda.synchronize()
-    rq_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) for lst in rq_ms]
-    gemm_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) for lst in gemm_ms]
+    rq_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in rq_ms]
+    gemm_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in gemm_ms]
     gemm_flops = sum(2.0 * M * K * N for (M, K, N) in shapes)
     gemm_tflops = gemm_flops / (sum(gemm_t) * 1e-3) / 1e12
     rq_bytes = sum(M * K * 2.53125 for (M, K, N) in shapes)
@@ -350,7 +372,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         rows = 256
-        prepared = oracle_prepare(shapes, cfg, rows, block)
+        prepared = oracle_prepare(shapes, cfg, rows, block, idx)
         t, f, passes = 0.0, 0.0, 0
         while t < 10.0 and passes < 200:          # about 10 s of CPU work
             dt, df = oracle_step(prepared, block)
@@ -374,6 +396,7 @@ def run_ours(args):
                          "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
                          "peak_source": f"{FP4_OVER_BF16:.0f} x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s)",
                          "traffic": None, "algorithmic_bytes": gemm_bytes,
+                         "timing": f"CUDA events around groups of {ring} back-to-back launches, {inst_steps} groups per shape",
                          "per_shape_us": [round(t * 1e3, 2) for t in gemm_t]},
             "rotate_quantize": {"bound": "hbm", "achieved": rq_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                 "frac": rq_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -455,6 +478,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--block", type=int, default=32)
+    ap.add_argument("--shape-index", type=int, default=-1,
+                    help="run only this shape of the workload (for profiling captures); -1 = all")
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="rows per shape per step for --impl reference (0 = sized to finish in ~2 min)")
     ap.add_argument("--only-block", action="store_true", help="cfg4: run only --block instead of the sweep")
