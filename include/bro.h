@@ -150,6 +150,40 @@ bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int bl
                            void* y_host_bf16, void* x_stage, void* y_stage, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/*
+ * bro_linear for callers that cannot hand over a workspace.  (The paper has no counterpart: this
+ * entry point exists for integration reasons only; the arithmetic is bro_linear's.)
+ *
+ * Who needs it: code that runs where device allocation is off limits — inside a region that is
+ * being captured into a CUDA graph by someone else, in a plugin whose host framework owns the
+ * allocator and gives the plugin only its input and output tensors, or in a serving loop that
+ * has pinned its memory budget and forbids cudaMalloc after start-up.  Such a caller has x, the
+ * packed weights and y, but nowhere to put the quantised activations that sit between the two
+ * kernels.  Here that intermediate lives in an array compiled into the library:
+ *   BRO_STATIC_SCRATCH_BYTES of device memory per GPU, reserved when the library is loaded on
+ *   that GPU and held until the process exits, whether or not this function is ever called.
+ * The function itself allocates nothing: no cudaMalloc/cudaFree, no allocating library call.
+ *
+ * Limit: align256(M*K/2) + bro_scales_bytes(M, K, BRO_LAYOUT_GEMM) + bro_gemm_workspace_bytes(M, N, K)
+ * must not exceed BRO_STATIC_SCRATCH_BYTES (about M*K <= 31 million elements); a larger
+ * problem returns BRO_ERR_WORKSPACE, launches nothing and leaves a one-line explanation in
+ * bro_last_cuda_error().  All other arguments, requirements and errors are those of bro_linear.
+ *
+ * Set-up: the first call on each device looks up the array's device address (the name the
+ * host code sees is only a handle, not an address a kernel could use) and opts the kernels in to
+ * their shared-memory sizes.  Make that first call with the device current and outside any
+ * stream capture.
+ *
+ * Sharing: every call on a device uses the same array and finds in it whatever the previous
+ * call left.  Each call rewrites everything it later reads (padding included), so stale contents
+ * are harmless — but two calls that can run at the same time on one GPU (different streams,
+ * different host threads) race on the array.  Keep calls on one stream, or order them yourself.
+ */
+#define BRO_STATIC_SCRATCH_BYTES ((size_t)16 << 20)
+bro_status bro_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                             const void* wcodes, const void* wscales, int64_t N, void* y_bf16,
+                             int64_t ldy, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

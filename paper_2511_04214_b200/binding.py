@@ -24,7 +24,7 @@ EXPORTS = [
     "bro_status_string", "bro_last_cuda_error", "bro_codes_bytes", "bro_scales_bytes", "bro_scale_offset",
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
-    "bro_linear_host",
+    "bro_linear_host", "bro_linear_static",
 ]
 
 
@@ -68,6 +68,8 @@ def _load() -> ctypes.CDLL:
     L.bro_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p, sz, p]
     L.bro_linear_host.restype = ci
     L.bro_linear_host.argtypes = [p, i64, i64, ci, p, p, i64, p, p, p, p, sz, p]
+    L.bro_linear_static.restype = ci
+    L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
     return L
 
 
@@ -179,3 +181,24 @@ def linear_host(x_host: torch.Tensor, block: int, wcodes, wscales, N: int, y_hos
     _check(lib.bro_linear_host(_ptr(x_host), M, K, block, _ptr(wcodes), _ptr(wscales), N,
                                _ptr(y_host), _ptr(x_stage), _ptr(y_stage), _ptr(workspace),
                                workspace.numel(), _stream(stream)), "bro_linear_host")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def linear_static(x: torch.Tensor, block: int, wcodes, wscales, N: int, y: torch.Tensor,
+                  stream=None) -> None:
+    """``linear`` for callers that may not allocate device memory (a plugin that only receives its
+    input and output tensors, code running while someone else captures a CUDA graph, a server that
+    forbids allocation after start-up): the quantised activations go to a ``STATIC_SCRATCH_BYTES``
+    array built into the library, so the problem must fit it (roughly M*K <= 31 million).  Calls
+    on one GPU share that array — keep them on one stream.  Make the first call per device outside
+    stream capture."""
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+    M, K = x.shape
+    code = lib.bro_linear_static(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K), block,
+                                 _ptr(wcodes), _ptr(wscales), N, _ptr(y),
+                                 y.stride(0) if M > 1 else max(y.stride(0), N), _stream(stream))
+    if code == 5:
+        raise BroError(code, "bro_linear_static: " + lib.bro_last_cuda_error().decode())
+    _check(code, "bro_linear_static")

@@ -307,4 +307,53 @@ bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int bl
   return BRO_OK;
 }
 
+// ---- bro_linear without a caller-provided workspace ---------------------------------------------
+// The quantised activations (and any GEMM workspace) live in this array instead.  In host code the
+// name is only a handle: the address a kernel can use comes from cudaGetSymbolAddress, looked up
+// once per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[BRO_STATIC_SCRATCH_BYTES];
+
+bro_status bro_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                             const void* wcodes, const void* wscales, int64_t N, void* y_bf16, int64_t ldy,
+                             void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (M == 0 || N == 0) return BRO_OK;
+  if (!x_bf16 || !wcodes || !wscales || !y_bf16) return BRO_ERR_NULL;
+  const size_t codes_sz = align_up(bro_codes_bytes(M, K), 256);
+  const size_t scales_sz = align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 256);
+  const size_t gemm_sz = bro_gemm_workspace_bytes(M, N, K);
+  const size_t need = codes_sz + scales_sz + gemm_sz;
+  if (need > BRO_STATIC_SCRATCH_BYTES) {
+    snprintf(bro::g_last_cuda_error, sizeof(bro::g_last_cuda_error),
+             "bro_linear_static: this problem needs %zu bytes of scratch, the built-in array holds %zu; "
+             "use bro_linear with a workspace", need, (size_t)BRO_STATIC_SCRATCH_BYTES);
+    return BRO_ERR_WORKSPACE;
+  }
+  // Device address of the array, once per device, with that device current.
+  static unsigned char* base_of[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  if (!bro::cuda_ok(cudaGetDevice(&dev), "cudaGetDevice")) return BRO_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return BRO_ERR_UNSUPPORTED;
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!base_of[dev]) {
+      void* p = nullptr;
+      if (!bro::cuda_ok(cudaGetSymbolAddress(&p, g_static_scratch), "cudaGetSymbolAddress(static scratch)") || !p)
+        return BRO_ERR_CUDA;
+      base_of[dev] = static_cast<unsigned char*>(p);
+    }
+    base = base_of[dev];
+  }
+  unsigned char* acodes = base;
+  unsigned char* ascales = acodes + codes_sz;
+  unsigned char* gws = ascales + scales_sz;
+  bro_status rc = bro_rotate_quantize_mxfp4(x_bf16, M, K, ldx, block, acodes, ascales, BRO_LAYOUT_GEMM, stream);
+  if (rc != BRO_OK) return rc;
+  return bro_gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16,
+                        gemm_sz ? gws : nullptr, gemm_sz, stream);
+}
+
 }  // extern "C"
