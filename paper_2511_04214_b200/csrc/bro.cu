@@ -10,6 +10,7 @@
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_global.cuh"
 #include "gemm_mxfp4.cuh"
+#include "gemm_mxfp4_2cta.cuh"
 
 namespace {
 
@@ -111,6 +112,15 @@ bro_status bro::gemm::make_out_map(CUtensorMap* map, const void* y, int64_t M, i
                      bro::gemm::kChunkCols, bro::gemm::kBM, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
+// Scale tensor in the tensor-core layout viewed as 32-bit words: one row per 128-row block
+// (kblocks * 512 bytes), box = one K step (1024 bytes) x box_rows row blocks, no swizzle.
+bro_status bro::gemm2::make_scale_map(CUtensorMap* map, const void* scales, int64_t rows, int64_t kblocks,
+                                      int box_rows) {
+  return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, scales, (uint64_t)(kblocks * 128),
+                     (uint64_t)ceil_div(rows, 128), (uint64_t)(kblocks * 512), 256, (uint32_t)box_rows,
+                     CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+
 namespace {
 
 // ---- rotate + quantise ---------------------------------------------------------------------------
@@ -163,8 +173,10 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
       if (r != BRO_OK) return r;
       attr_done[dev][which] = true;
     }
-    kernel<<<grid, bro::rq::kThreads, bro::rq::kSmemBytes, st>>>(tmx, p);
-    return bro::cuda_ok(cudaGetLastError(), "rotate_quantize launch") ? BRO_OK : BRO_ERR_CUDA;
+    return bro::cuda_ok(bro::launch_kernel(kernel, (unsigned)grid, bro::rq::kThreads, bro::rq::kSmemBytes, st, 1, tmx, p),
+                        "rotate_quantize launch")
+               ? BRO_OK
+               : BRO_ERR_CUDA;
   };
   switch (B) {
     case 32: return go(bro::rq::rotate_quantize_kernel<5>, 0);
@@ -267,6 +279,13 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
   DeviceInfo di;
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
+  // Default: one CTA per 128 x BN tile.  BRO_GEMM_PAIR=1 selects the two-CTA kernel (256 x 256
+  // tiles, cta_group::2), which moves a third fewer bytes from L2 but measured no faster.
+  bool pair = false;
+  if (const char* e = getenv("BRO_GEMM_PAIR")) pair = atoi(e) != 0;
+  if (pair)
+    return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, di.sm_count,
+                              static_cast<cudaStream_t>(stream));
   return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,
                            workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream));
 }

@@ -19,6 +19,32 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
   return false;
 }
 
+// Launch with programmatic dependent launch enabled (and, if cluster_x > 1, that cluster width).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                 cudaStream_t st, unsigned cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // One status word per device (each device that loads the module gets its own instance).
 // 0 = OK; otherwise (BRO_ERR_TIMEOUT) | (site << 8).  Kernels only ever move it away from 0.
 __device__ unsigned int g_device_status = 0u;
@@ -97,6 +123,17 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
       : "memory");
+}
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel of the library is launched with the "programmatic stream serialization" attribute,
+// so the next kernel in the stream may be scheduled while this one still runs: its CTAs start on
+// SMs as they become free and run their prologue (barrier set-up, TMEM allocation, descriptor
+// prefetch) early.  griddep_wait() blocks until all earlier grids in the stream have completed
+// and their writes are visible; every thread calls it before its first access to global memory.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {

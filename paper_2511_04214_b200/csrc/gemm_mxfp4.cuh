@@ -78,19 +78,69 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// ---- issuing tensor-core work --------------------------------------------------------------------
+// The issuing warp runs its loop with all 32 lanes converged, so that addresses, descriptors and
+// loop counters stay warp-uniform: the tensor-core instructions take their operands from uniform
+// registers, and values computed under a divergent branch (or derived from something the compiler
+// cannot prove uniform, such as a raw threadIdx or a shared-memory load) have to cross register
+// files one by one, which makes instruction issue, not the tensor pipe, the limit.  One lane
+// executes the instruction itself: every wrapper below predicates it on `issue` (non-zero in that lane).
+// CG = 1: this CTA alone; CG = 2: the CTA pair (cta_group::2), issued by the leader CTA.
+template <int CG>
+__device__ __forceinline__ void tc_commit(uint32_t issue, uint32_t bar) {
+  if constexpr (CG == 1)
+    asm volatile(
+        "{ .reg .pred q; setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0]; }" ::"r"(bar),
+        "r"(issue)
+        : "memory");
+  else   // arrives on the barrier at this offset in both CTAs of the pair
+    asm volatile(
+        "{ .reg .pred q; setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %2; }" ::"r"(bar),
+        "r"(issue), "h"((uint16_t)3)
+        : "memory");
 }
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+// Descriptors are passed as their two 32-bit halves: the upper half is a constant per descriptor
+// kind, the lower half is base + a small offset, so no 64-bit arithmetic is needed per instruction.
+template <int CG>
+__device__ __forceinline__ void tc_cp_sf(uint32_t issue, uint32_t taddr, uint32_t desc_lo, uint32_t desc_hi) {
+  if constexpr (CG == 1)
+    asm volatile(
+        "{ .reg .pred q; .reg .b64 d; setp.ne.b32 q, %3, 0; mov.b64 d, {%1, %2};\n\t"
+        "@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], d; }" ::"r"(taddr),
+        "r"(desc_lo), "r"(desc_hi), "r"(issue)
+        : "memory");
+  else
+    asm volatile(
+        "{ .reg .pred q; .reg .b64 d; setp.ne.b32 q, %3, 0; mov.b64 d, {%1, %2};\n\t"
+        "@q tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], d; }" ::"r"(taddr),
+        "r"(desc_lo), "r"(desc_hi), "r"(issue)
+        : "memory");
 }
-__device__ __forceinline__ void tc_mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile(
-      "{ .reg .pred p; setp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p; }" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
-      : "memory");
+template <int CG>
+__device__ __forceinline__ void tc_mma_mxf4(uint32_t issue, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                            uint32_t desc_hi, uint32_t idesc, uint32_t sfa_tmem, uint32_t sfb_tmem,
+                                            uint32_t accumulate) {
+  if constexpr (CG == 1)
+    asm volatile(
+        "{ .reg .pred p, q; .reg .b64 da, db; setp.ne.b32 p, %7, 0; setp.ne.b32 q, %8, 0;\n\t"
+        "mov.b64 da, {%1, %3}; mov.b64 db, {%2, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %4, [%5], [%6], p; }" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate), "r"(issue)
+        : "memory");
+  else
+    asm volatile(
+        "{ .reg .pred p, q; .reg .b64 da, db; setp.ne.b32 p, %7, 0; setp.ne.b32 q, %8, 0;\n\t"
+        "mov.b64 da, {%1, %3}; mov.b64 db, {%2, %3};\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %4, [%5], [%6], p; }" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate), "r"(issue)
+        : "memory");
+}
+// Bounded wait executed by a whole converged warp; the result is the same in every lane.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned site) {
+  const bool ok = mbar_wait(bar, parity, site);
+  return __all_sync(0xFFFFFFFFu, ok);
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -107,24 +157,15 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 
 // ---- descriptors -------------------------------------------------------------------------------
 // Shared-memory matrix descriptor, K-major operand stored as rows of 128 bytes with the 128-byte
-// swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);   // start address / 16
-  d |= (uint64_t)1 << 16;                   // leading byte offset / 16 (unused with swizzle)
-  d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset / 16
-  d |= (uint64_t)1 << 46;                   // descriptor version (sm_100)
-  d |= (uint64_t)2 << 61;                   // layout: 128-byte swizzle
-  return d;
-}
+// swizzle (8-row groups 1024 bytes apart).  Low word: start address / 16 in bits 0..13, leading
+// byte offset / 16 = 1 in bits 16..29 (unused with swizzle).  High word: stride byte offset / 16
+// in bits 0..13, descriptor version 1 in bit 14, layout 2 (128-byte swizzle) in bits 29..31.
+// Advancing by 64 K elements (32 bytes) inside the swizzled row adds 2 to the low word.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t saddr) { return ((saddr >> 4) & 0x3FFFu) | (1u << 16); }
 // Scale block: 32 rows x 16 bytes, dense, no swizzle; 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sf(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)(128 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  return d;
-}
+constexpr uint32_t kDescHiSf = (128u >> 4) | (1u << 14);
+__device__ __forceinline__ uint32_t desc_lo_sf(uint32_t saddr) { return (saddr >> 4) & 0x3FFFu; }
 // Instruction descriptor, kind::mxf4 block-scaled: E2M1 x E2M1, both K-major, UE8M0 scales,
 // dense K = 64, M x N = 128 x BN; scale-factor byte ids filled in per K block.
 template <int BN>
@@ -165,6 +206,86 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// Addresses the issuing warp works with (shared-memory window addresses of stage 0 and of the
+// first barrier of each kind).
+struct IssueRing {
+  uint32_t sA, sB, sSFA, sSFB;
+  uint32_t bar_full, bar_empty, bar_acc_full, bar_acc_free, bar_ovl_free;
+};
+
+// The K loop of the issuing warp over all tiles of this CTA (or CTA pair), shared by both kernels.
+// Per 256-element K step: two scale-block copies shared -> TMEM per operand row block and four
+// MMAs of K = 64.  The two 128-element halves of a step own separate TMEM scale columns
+// (A: 4 columns at 4h; W: BN/32 columns at (BN/32)h), and the copies for the NEXT step are issued
+// between the halves of the current one, so a copy never sits directly in front of its consumer.
+// Accumulator t & 1 is used for this CTA's t-th tile; with OVERLAP the two accumulators share
+// columns that the epilogue of the other buffer releases through bar_ovl_free.
+template <int CG, int BN, int STAGES, int A_STAGE, int B_STAGE, int SFA_STAGE, int SFB_STAGE, int ACC_STRIDE,
+          bool OVERLAP>
+__device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem_base, uint32_t tmem_sfa,
+                                               uint32_t tmem_sfb, uint32_t idesc0, int my_tiles, int num_k_steps,
+                                               bool issue_lane) {
+  const uint32_t issue = issue_lane ? 1u : 0u;
+  const uint32_t a_lo0 = desc_lo_sw128(r.sA), b_lo0 = desc_lo_sw128(r.sB);
+  const uint32_t sfa_lo0 = desc_lo_sf(r.sSFA), sfb_lo0 = desc_lo_sf(r.sSFB);
+  const uint32_t hi_op = kDescHiSw128, hi_sf = kDescHiSf;
+  // scale bytes {0,1} of a 32-bit scale word for the first MMA of a half, {2,3} for the second
+  const uint32_t idesc1 = idesc0 | (2u << 4) | (2u << 29);
+  auto copy_scales = [&](int stage, int h) {
+    const uint32_t lo_a = sfa_lo0 + (uint32_t)stage * (SFA_STAGE >> 4) + (uint32_t)h * 32u;
+    const uint32_t lo_b = sfb_lo0 + (uint32_t)stage * (SFB_STAGE >> 4) + (uint32_t)h * 32u;
+    tc_cp_sf<CG>(issue, tmem_sfa + 4 * h, lo_a, hi_sf);
+#pragma unroll
+    for (int nb = 0; nb < BN / 128; ++nb) tc_cp_sf<CG>(issue, tmem_sfb + (BN / 32) * h + 4 * nb, lo_b + 64u * nb, hi_sf);
+  };
+  auto mma_half = [&](int stage, int h, uint32_t tmem_acc, uint32_t accumulate_first) {
+    const uint32_t a_lo = a_lo0 + (uint32_t)stage * (A_STAGE >> 4) + 4u * h;
+    const uint32_t b_lo = b_lo0 + (uint32_t)stage * (B_STAGE >> 4) + 4u * h;
+    const uint32_t tsfa = tmem_sfa + 4 * h, tsfb = tmem_sfb + (BN / 32) * h;
+    tc_mma_mxf4<CG>(issue, tmem_acc, a_lo, b_lo, hi_op, idesc0, tsfa, tsfb, accumulate_first);
+    tc_mma_mxf4<CG>(issue, tmem_acc, a_lo + 2u, b_lo + 2u, hi_op, idesc1, tsfa | (2u << 30), tsfb | (2u << 30), 1u);
+  };
+  int stage = 0;
+  uint32_t phase = 0;
+  bool ok = my_tiles > 0;
+  if (ok) ok = mbar_wait_warp(r.bar_full, 0u, SITE_GEMM_FULL);
+  if (ok) {
+    tc_fence_after();
+    copy_scales(0, 0);
+    copy_scales(0, 1);
+  }
+  for (int it = 0; it < my_tiles && ok; ++it) {
+    const int buf = it & 1;
+    const int use = it >> 1;                       // how many times this buffer was used before
+    // this buffer must have been drained by the epilogue of tile it-2 ...
+    if (use >= 1) ok = mbar_wait_warp(r.bar_acc_free + 8 * buf, (uint32_t)((use - 1) & 1), SITE_GEMM_ACC_EMPTY);
+    // ... and the columns it shares with the other buffer by the epilogue of tile it-1
+    if (ok && OVERLAP && it >= 1)
+      ok = mbar_wait_warp(r.bar_ovl_free + 8 * (buf ^ 1), (uint32_t)(((it - 1) >> 1) & 1), SITE_GEMM_ACC_EMPTY);
+    if (!ok) break;
+    tc_fence_after();
+    const uint32_t tmem_acc = tmem_base + buf * ACC_STRIDE;
+    for (int ks = 0; ks < num_k_steps; ++ks) {
+      const bool has_next = (ks + 1 < num_k_steps) || (it + 1 < my_tiles);
+      const int next_stage = (stage + 1 == STAGES) ? 0 : stage + 1;
+      const uint32_t next_phase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
+      mma_half(stage, 0, tmem_acc, ks == 0 ? 0u : 1u);
+      if (has_next) {
+        ok = mbar_wait_warp(r.bar_full + 8 * next_stage, next_phase, SITE_GEMM_FULL);
+        if (!ok) break;
+        tc_fence_after();
+        copy_scales(next_stage, 0);          // half 0's columns were last read by the two MMAs above
+      }
+      mma_half(stage, 1, tmem_acc, 1u);
+      tc_commit<CG>(issue, r.bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
+      if (has_next) copy_scales(next_stage, 1);
+      stage = next_stage;
+      phase = next_phase;
+    }
+    tc_commit<CG>(issue, r.bar_acc_full + 8 * buf);    // accumulator complete (or abandoned) -> epilogue
+  }
+}
+
 template <int BN, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw,
@@ -186,7 +307,9 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   const uint32_t tmem_slot = bar_ovl_free + 16;                    // u32 written by tcgen05.alloc
   uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
-  const int warp = threadIdx.x >> 5;
+  // (the shuffle tells the compiler that the warp index is the same in all lanes, so that role
+  // branches and everything computed under them can use the uniform datapath)
+  const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -209,7 +332,9 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot_ptr;
+  griddep_launch_dependents();
+  griddep_wait();               // operands come from the kernel before; y may still be read by it
+  const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot_ptr, 0);
   const uint32_t tmem_sfa = tmem_base + C::kSfaCol;
   const uint32_t tmem_sfb = tmem_base + C::kSfbCol;
 
@@ -251,53 +376,12 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc0 = make_idesc<BN>();
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      int it = 0;   // index of this CTA's tile
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++it) {
-        const int buf = it & 1;
-        const int use = it >> 1;                       // how many times this buffer was used before
-        // this buffer must have been drained by the epilogue of tile it-2 ...
-        if (use >= 1) ok = mbar_wait(bar_acc_free + 8 * buf, (uint32_t)((use - 1) & 1), SITE_GEMM_ACC_EMPTY);
-        // ... and the columns it shares with the other buffer by the epilogue of tile it-1
-        if (ok && C::kOverlap && it >= 1)
-          ok = mbar_wait(bar_ovl_free + 8 * (buf ^ 1), (uint32_t)(((it - 1) >> 1) & 1), SITE_GEMM_ACC_EMPTY);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t tmem_acc = tmem_base + buf * C::kAccStride;
-        for (int ks = 0; ks < p.num_k_steps; ++ks) {
-          ok = mbar_wait(bar_full + 8 * stage, phase, SITE_GEMM_FULL);
-          if (!ok) break;
-          tc_fence_after();
-          // scale blocks of this K step: shared -> TMEM.  K-block pair a (128 elements) of A goes to
-          // columns 4a..4a+3; of W to columns (BN/32)*a + 4*nb .. +3.
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            tc_cp_sf(tmem_sfa + 4 * a, smem_desc_sf(sSFA + stage * C::kSfaBytes + a * 512));
-#pragma unroll
-            for (int nb = 0; nb < BN / 128; ++nb)
-              tc_cp_sf(tmem_sfb + (BN / 32) * a + 4 * nb,
-                       smem_desc_sf(sSFB + stage * C::kSfbBytes + nb * 1024 + a * 512));
-          }
-          const uint64_t adesc = smem_desc_sw128(sA + stage * kATileBytes);
-          const uint64_t bdesc = smem_desc_sw128(sB + stage * C::kBTileBytes);
-#pragma unroll
-          for (int kb = 0; kb < 4; ++kb) {
-            const uint32_t sf_id = (kb & 1) * 2;          // bytes {0,1} or {2,3} of the scale word
-            const uint32_t idesc = idesc0 | (sf_id << 4) | (sf_id << 29);
-            const uint32_t tsfa = (tmem_sfa + 4 * (kb >> 1)) | (sf_id << 30);
-            const uint32_t tsfb = (tmem_sfb + (BN / 32) * (kb >> 1)) | (sf_id << 30);
-            tc_mma_mxf4(tmem_acc, adesc + 2 * kb, bdesc + 2 * kb, idesc, tsfa, tsfb, (ks | kb) != 0 ? 1u : 0u);
-          }
-          tc_commit(bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
-          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
-        }
-        tc_commit(bar_acc_full + 8 * buf);    // accumulator complete (or abandoned) -> epilogue
-      }
-    }
+    const IssueRing ring = {sA, sB, sSFA, sSFB, bar_full, bar_empty, bar_acc_full, bar_acc_free, bar_ovl_free};
+    const int my_tiles =
+        (int)blockIdx.x < p.total_tiles ? (p.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    mma_issue_loop<1, BN, C::kStages, kATileBytes, C::kBTileBytes, C::kSfaBytes, C::kSfbBytes, C::kAccStride,
+                   C::kOverlap>(ring, tmem_base, tmem_sfa, tmem_sfb, make_idesc<BN>(), my_tiles, p.num_k_steps,
+                                lane == 0);
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
@@ -407,8 +491,10 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
         return BRO_ERR_CUDA;
       attr_done[dev][which] = true;
     }
-    kernel<<<grid, kThreads, C::kSmemBytes, st>>>(tma, tmw, tmy, p);
-    return cuda_ok(cudaGetLastError(), "gemm_mxfp4 launch") ? BRO_OK : BRO_ERR_CUDA;
+    return cuda_ok(launch_kernel(kernel, (unsigned)grid, kThreads, C::kSmemBytes, st, 1, tma, tmw, tmy, p),
+                   "gemm_mxfp4 launch")
+               ? BRO_OK
+               : BRO_ERR_CUDA;
   };
   return out_dtype == BRO_OUT_F32 ? go(gemm_mxfp4_kernel<BN, true>, 1) : go(gemm_mxfp4_kernel<BN, false>, 0);
 }

@@ -37,6 +37,8 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   const uint32_t cbits = (p.log2k % 2 == 0) ? (uint32_t)(127 - p.log2k / 2) << 23
                                             : 0x3FB504F3u - ((uint32_t)((p.log2k + 1) / 2) << 23);
   const int64_t row_iters = (p.M + p.rows_per_iter - 1) / p.rows_per_iter;
+  griddep_launch_dependents();
+  griddep_wait();               // x may be written, codes/scales still read, by the kernel before
 
   for (int64_t it = blockIdx.x; it < row_iters; it += gridDim.x) {
     const int64_t row = it * p.rows_per_iter + rs;
@@ -127,8 +129,10 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, void*
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return BRO_ERR_CUDA;
-    kernel<<<grid, threads, smem, st>>>(p);
-    return cuda_ok(cudaGetLastError(), "rotate_quantize_global launch") ? BRO_OK : BRO_ERR_CUDA;
+    return cuda_ok(launch_kernel(kernel, (unsigned)grid, (unsigned)threads, smem, st, 1, p),
+                   "rotate_quantize_global launch")
+               ? BRO_OK
+               : BRO_ERR_CUDA;
   };
   if (threads <= 256) return go(rotate_quantize_global_kernel<256>);
   if (threads <= 512) return go(rotate_quantize_global_kernel<512>);

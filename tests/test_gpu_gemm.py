@@ -77,15 +77,22 @@ def quantized_pair(M, N, K, seed, block=32, recipe=synth.HEAVY_RECIPE):
     return x, w, ac, asc, wc, wsc
 
 
-@pytest.fixture(params=["128", "256"])
+@pytest.fixture(params=["cta1_n128", "cta1_n256", "pair"])
 def tile_n(request):
-    old = os.environ.get("BRO_GEMM_TILE_N")
-    os.environ["BRO_GEMM_TILE_N"] = request.param
-    yield int(request.param)
-    if old is None:
-        del os.environ["BRO_GEMM_TILE_N"]
+    """Force each GEMM kernel variant in turn: the single-CTA kernel with 128- or 256-column tiles,
+    and the two-CTA (cta_group::2) kernel with 256 x 256 tiles."""
+    saved = {k: os.environ.get(k) for k in ("BRO_GEMM_TILE_N", "BRO_GEMM_PAIR")}
+    if request.param == "pair":
+        os.environ["BRO_GEMM_PAIR"] = "1"
     else:
-        os.environ["BRO_GEMM_TILE_N"] = old
+        os.environ["BRO_GEMM_PAIR"] = "0"
+        os.environ["BRO_GEMM_TILE_N"] = request.param[-3:]
+    yield request.param
+    for k, v in saved.items():
+        if v is None:
+            os.environ.pop(k, None)
+        else:
+            os.environ[k] = v
 
 
 def test_unit_scales_small_integers_exact(bro, tile_n):
@@ -126,7 +133,7 @@ def test_config1_full_output(bro, tile_n):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (129, 136, 160), (300, 520, 416), (128, 256, 288),
-                                   (257, 129, 1024), (64, 384, 3072)])
+                                   (257, 129, 1024), (64, 384, 3072), (700, 1300, 512), (2304, 1000, 768)])
 def test_ragged_shapes(bro, tile_n, M, N, K):
     _, _, ac, asc, wc, wsc = quantized_pair(M, N, K, seed=M + N + K)
     run_case(bro, ac, asc, wc, wsc)
