@@ -136,6 +136,38 @@ __device__ __forceinline__ void griddep_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Forms for a converged warp in which one lane issues: `issue` is non-zero in that lane only.  The
+// loop around them, and every address they take, stays warp-uniform.
+__device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t issue, uint32_t bar, uint32_t bytes) {
+  asm volatile(
+      "{ .reg .pred q; .reg .b64 st; setp.ne.b32 q, %2, 0;\n\t"
+      "@q mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar),
+      "r"(bytes), "r"(issue)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, int x, int y,
+                                               uint32_t bar) {
+  asm volatile(
+      "{ .reg .pred q; setp.ne.b32 q, %5, 0;\n\t"
+      "@q cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4]; }" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar), "r"(issue)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load_1d_if(uint32_t issue, uint32_t dst, const void* src, uint32_t bytes,
+                                                uint32_t bar) {
+  asm volatile(
+      "{ .reg .pred q; setp.ne.b32 q, %4, 0;\n\t"
+      "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3]; }" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "r"(issue)
+      : "memory");
+}
+// Bounded wait executed by a whole converged warp; the result is the same in every lane.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned site) {
+  const bool ok = mbar_wait(bar, parity, site);
+  return __all_sync(0xFFFFFFFFu, ok);
+}
+
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"

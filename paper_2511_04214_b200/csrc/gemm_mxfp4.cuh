@@ -137,11 +137,6 @@ __device__ __forceinline__ void tc_mma_mxf4(uint32_t issue, uint32_t d_tmem, uin
         "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate), "r"(issue)
         : "memory");
 }
-// Bounded wait executed by a whole converged warp; the result is the same in every lane.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, unsigned site) {
-  const bool ok = mbar_wait(bar, parity, site);
-  return __all_sync(0xFFFFFFFFu, ok);
-}
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -269,9 +264,13 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
       const bool has_next = (ks + 1 < num_k_steps) || (it + 1 < my_tiles);
       const int next_stage = (stage + 1 == STAGES) ? 0 : stage + 1;
       const uint32_t next_phase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
+      // Probe the next stage's barrier before issuing: the answer travels while the two MMAs
+      // below are issued, and in the steady state it is "ready", so the issuing warp rarely
+      // spends a barrier round trip between tensor-core instructions.
+      const bool probe = has_next && mbar_try_wait(r.bar_full + 8 * next_stage, next_phase);
       mma_half(stage, 0, tmem_acc, ks == 0 ? 0u : 1u);
       if (has_next) {
-        ok = mbar_wait_warp(r.bar_full + 8 * next_stage, next_phase, SITE_GEMM_FULL);
+        if (!__all_sync(0xFFFFFFFFu, probe)) ok = mbar_wait_warp(r.bar_full + 8 * next_stage, next_phase, SITE_GEMM_FULL);
         if (!ok) break;
         tc_fence_after();
         copy_scales(next_stage, 0);          // half 0's columns were last read by the two MMAs above

@@ -75,12 +75,13 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 }
 // 2-D tiled load into THIS CTA's shared memory whose byte count completes on an mbarrier that may
 // live in the partner CTA (shared::cluster address).  No multicast.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, int x, int y,
-                                                 uint32_t bar_cluster) {
+__device__ __forceinline__ void tma_load_2d_pair_if(uint32_t issue, uint32_t dst, const CUtensorMap* m, int x,
+                                                    int y, uint32_t bar_cluster) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar_cluster)
+      "{ .reg .pred q; setp.ne.b32 q, %5, 0;\n\t"
+      "@q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4]; }" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar_cluster), "r"(issue)
       : "memory");
 }
 // E2M1 x E2M1, K-major, UE8M0 scales, M = 256 (128 rows per CTA), N = 256.
@@ -157,30 +158,35 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
 
   if (warp == 0) {
     // ------------------------------ TMA producer (both CTAs) ------------------------------
-    if (lane == 0) {
-      tma_prefetch_desc(&tma);
-      tma_prefetch_desc(&tmw);
-      tma_prefetch_desc(&tmsfa);
-      tma_prefetch_desc(&tmsfb);
+    // All 32 lanes walk the loop together (uniform addresses and counters); lane 0 issues.
+    {
+      const uint32_t issue = lane == 0 ? 1u : 0u;
+      if (lane == 0) {
+        tma_prefetch_desc(&tma);
+        tma_prefetch_desc(&tmw);
+        tma_prefetch_desc(&tmsfa);
+        tma_prefetch_desc(&tmsfb);
+      }
       int stage = 0;
       uint32_t phase = 0;
       int64_t issued = 0;
       bool ok = true;
+      const uint32_t full0 = map_to_cta(bar_full, 0);      // the leader's barriers, as seen from here
       for (int tile = pair; tile < p.total_tiles && ok; tile += num_pairs) {
         int tm, tn;
         tile_coords(tile, p, tm, tn);
         const int m0 = tm * 256 + (int)rank * kBM;
         const int n0 = tn * kBN;
         for (int ks = 0; ks < p.num_k_steps; ++ks) {
-          if (issued >= kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
+          if (issued >= kStages) ok = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
           if (!ok) break;
-          if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * kStageBytes);
-          const uint32_t full = map_to_cta(bar_full + 8 * stage, 0);
-          tma_load_2d_pair(sA + stage * kATileBytes, &tma, ks * 128, m0, full);
-          tma_load_2d_pair(sB + stage * kBTileBytes, &tmw, ks * 128, n0 + (int)rank * (kBN / 2), full);
+          if (rank == 0) mbar_arrive_expect_tx_if(issue, bar_full + 8 * stage, 2 * kStageBytes);
+          const uint32_t full = full0 + 8 * stage;
+          tma_load_2d_pair_if(issue, sA + stage * kATileBytes, &tma, ks * 128, m0, full);
+          tma_load_2d_pair_if(issue, sB + stage * kBTileBytes, &tmw, ks * 128, n0 + (int)rank * (kBN / 2), full);
           // scale maps are in 32-bit elements: one K step = 1024 bytes = 256 elements per row block
-          tma_load_2d_pair(sSFA + stage * kSfaBytes, &tmsfa, ks * 256, m0 >> 7, full);
-          tma_load_2d_pair(sSFB + stage * kSfbBytes, &tmsfb, ks * 256, n0 >> 7, full);
+          tma_load_2d_pair_if(issue, sSFA + stage * kSfaBytes, &tmsfa, ks * 256, m0 >> 7, full);
+          tma_load_2d_pair_if(issue, sSFB + stage * kSfbBytes, &tmsfb, ks * 256, n0 >> 7, full);
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -190,7 +196,7 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
         // armed on every stage.  The partner's copies are counted on the same barriers.
         const int64_t first = issued > kStages ? issued - kStages : 0;
         for (int64_t i = first; i < issued; ++i)
-          mbar_wait(bar_full + 8 * (int)(i % kStages), (uint32_t)((i / kStages) & 1), SITE_GEMM_DRAIN);
+          mbar_wait_warp(bar_full + 8 * (int)(i % kStages), (uint32_t)((i / kStages) & 1), SITE_GEMM_DRAIN);
       }
     }
   } else if (warp == 1) {
