@@ -59,6 +59,23 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(value, dist, device):
+    """The largest `value` over all ranks of the job (the job's time is its slowest rank's)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_rank_per_step, steps, world, ms_max):
+    """Whole-job throughput: every rank runs an independent replica of the workload (weak scaling,
+    no exchange on the data path), so the job processed world * steps * units in the time of the
+    slowest rank."""
+    return units_per_rank_per_step * steps * world / (ms_max * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the GPU works."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -280,15 +297,11 @@ def run_ours(args):
     e1.record()
     barrier()
     sampler.mark("t1")
-    ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     status = bro.last_device_status()
     if status != 0:
         raise SystemExit(f"device status {bro.status_string(status)} after the timed region")
-    value = flops_per_step * steps * world / (ms_total * 1e-3) / 1e12
+    value = aggregate_throughput(flops_per_step, steps, world, ms_total) / 1e12
 
     # ---- instrumented pass for the per-kernel roofline: the two C-ABI calls bro_linear makes,
     # each timed with CUDA events around a group of `ring` back-to-back launches (one per ring
@@ -356,12 +369,8 @@ def run_ours(args):
             e2e_step()
         b.record()
         barrier()
-        ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": flops_per_step * n_e2e * world / (ms * 1e-3) / 1e12, "unit": UNIT,
+        ms = max_over_ranks(a.elapsed_time(b), dist, dev)
+        e2e = {"value": aggregate_throughput(flops_per_step, n_e2e, world, ms) / 1e12, "unit": UNIT,
                "h2d_bytes_per_step": sum(M * K * 2 for (M, K, N) in shapes),
                "d2h_bytes_per_step": sum(M * N * 2 for (M, K, N) in shapes), "steps": n_e2e}
 
