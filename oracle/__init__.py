@@ -45,6 +45,8 @@ def lib() -> ctypes.CDLL:
         L.bro_ref_hadamard_norm.restype = ctypes.c_float
         L.bro_ref_hadamard_norm.argtypes = [i64]
         L.bro_ref_rotate.argtypes = [p, i64, i64, i64, ci, p]
+        L.bro_ref_rotate_rs.argtypes = [p, i64, i64, i64, ci, p, p]
+        L.bro_ref_rotate_quantize_mxfp4_rs.argtypes = [p, i64, i64, i64, ci, p, p, p]
         L.bro_ref_quantize.argtypes = [p, i64, i64, p, p]
         L.bro_ref_decode.argtypes = [p, p, i64, i64, p]
         L.bro_ref_rotate_quantize_mxfp4.argtypes = [p, i64, i64, i64, ci, p, p]
@@ -53,7 +55,7 @@ def lib() -> ctypes.CDLL:
         L.bro_ref_gemm_mxfp4_points.argtypes = [p, p, p, p, i64, i64, i64, p, p, i64, p, p]
         L.bro_ref_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, p]
         L.bro_ref_group_mse.argtypes = [p, p, p, i64, i64, p]
-        for name in ("rotate", "quantize", "decode", "rotate_quantize_mxfp4", "pack_weights",
+        for name in ("rotate_rs", "rotate_quantize_mxfp4_rs", "rotate", "quantize", "decode", "rotate_quantize_mxfp4", "pack_weights",
                      "gemm_mxfp4", "gemm_mxfp4_points", "linear", "group_mse"):
             getattr(L, "bro_ref_" + name).restype = ci
         _lib = L
@@ -90,11 +92,24 @@ def hadamard_norm(block: int) -> np.float32:
     return np.float32(lib().bro_ref_hadamard_norm(int(block)))
 
 
-def rotate(x_bits, block: int) -> np.ndarray:
+def _signs(signs_bits, K: int):
+    if signs_bits is None:
+        return None
+    s = np.ascontiguousarray(signs_bits)
+    if s.dtype != np.uint16 or s.shape != (K,):
+        raise TypeError("signs are passed as a uint16 [K] array of bf16 bit patterns (+1 / -1)")
+    return s
+
+
+def rotate(x_bits, block: int, signs_bits=None) -> np.ndarray:
+    """Rotation only.  ``signs_bits`` ([K] bf16 bit patterns of +-1) selects the randomised form
+    R_i = diag(s) H / sqrt(block); None is the plain normalised Hadamard."""
     x = _as_bf16_bits(x_bits)
     M, K = x.shape
     y = np.empty((M, K), dtype=np.float32)
-    _check(lib().bro_ref_rotate(_ptr(x), M, K, K, int(block), _ptr(y)), "rotate")
+    s = _signs(signs_bits, K)
+    _check(lib().bro_ref_rotate_rs(_ptr(x), M, K, K, int(block), None if s is None else _ptr(s),
+                                   _ptr(y)), "rotate_rs")
     return y
 
 
@@ -116,17 +131,21 @@ def decode(codes, scales) -> np.ndarray:
     return out
 
 
-def rotate_quantize_mxfp4(x_bits, block: int) -> tuple[np.ndarray, np.ndarray]:
+def rotate_quantize_mxfp4(x_bits, block: int, signs_bits=None) -> tuple[np.ndarray, np.ndarray]:
     x = _as_bf16_bits(x_bits)
     M, K = x.shape
     codes = np.empty((M, K // 2), dtype=np.uint8)
     scales = np.empty((M, K // MX_GROUP), dtype=np.uint8)
-    _check(lib().bro_ref_rotate_quantize_mxfp4(_ptr(x), M, K, K, int(block), _ptr(codes),
-                                               _ptr(scales)), "rotate_quantize_mxfp4")
+    s = _signs(signs_bits, K)
+    _check(lib().bro_ref_rotate_quantize_mxfp4_rs(_ptr(x), M, K, K, int(block),
+                                                  None if s is None else _ptr(s), _ptr(codes),
+                                                  _ptr(scales)), "rotate_quantize_mxfp4_rs")
     return codes, scales
 
 
-def pack_weights(w_bits, block: int) -> tuple[np.ndarray, np.ndarray]:
+def pack_weights(w_bits, block: int, signs_bits=None) -> tuple[np.ndarray, np.ndarray]:
+    if signs_bits is not None:           # the same arithmetic on the rows of W, same sign vector
+        return rotate_quantize_mxfp4(w_bits, block, signs_bits)
     w = _as_bf16_bits(w_bits)
     N, K = w.shape
     codes = np.empty((N, K // 2), dtype=np.uint8)
@@ -167,7 +186,10 @@ def gemm_mxfp4_points(acodes, ascales, wcodes, wscales, pm, pn) -> tuple[np.ndar
     return y, S
 
 
-def linear(x_bits, block: int, wcodes, wscales) -> tuple[np.ndarray, np.ndarray]:
+def linear(x_bits, block: int, wcodes, wscales, signs_bits=None) -> tuple[np.ndarray, np.ndarray]:
+    if signs_bits is not None:
+        ac, asc = rotate_quantize_mxfp4(x_bits, block, signs_bits)
+        return gemm_mxfp4(ac, asc, wcodes, wscales)
     x = _as_bf16_bits(x_bits)
     wcodes = np.ascontiguousarray(wcodes, dtype=np.uint8)
     wscales = np.ascontiguousarray(wscales, dtype=np.uint8)

@@ -77,7 +77,8 @@ static void fwht_block(float* v, int64_t B) {
   }
 }
 
-int bro_ref_rotate(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int block, float* y) {
+int bro_ref_rotate_rs(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int block,
+                      const uint16_t* signs, float* y) {
   if (!x || !y) return 1;
   if (M < 0 || K <= 0 || ldx < K) return 2;
   int64_t B = block == 0 ? K : block;
@@ -86,13 +87,22 @@ int bro_ref_rotate(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int blo
 #pragma omp parallel for schedule(static)
   for (int64_t m = 0; m < M; ++m) {
     float* row = y + m * K;
-    for (int64_t k = 0; k < K; ++k) row[k] = bf16_to_f32(x[m * ldx + k]);
+    for (int64_t k = 0; k < K; ++k) {
+      float v = bf16_to_f32(x[m * ldx + k]);
+      /* x diag(s): channel k is negated where s_k = -1 (exact) */
+      if (signs && (signs[k] & 0x8000u)) v = -v;
+      row[k] = v;
+    }
     for (int64_t b0 = 0; b0 < K; b0 += B) {
       fwht_block(row + b0, B);
       for (int64_t i = 0; i < B; ++i) row[b0 + i] = row[b0 + i] * c; /* one multiply, at the end */
     }
   }
   return 0;
+}
+
+int bro_ref_rotate(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int block, float* y) {
+  return bro_ref_rotate_rs(x, M, K, ldx, block, NULL, y);
 }
 
 /* Round a non-negative scaled magnitude r onto the E2M1 grid, nearest, ties to the even code,
@@ -167,17 +177,23 @@ int bro_ref_decode(const uint8_t* codes, const uint8_t* scales, int64_t rows, in
   return 0;
 }
 
-int bro_ref_rotate_quantize_mxfp4(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
-                                  int block, uint8_t* codes, uint8_t* scales) {
+int bro_ref_rotate_quantize_mxfp4_rs(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
+                                     int block, const uint16_t* signs, uint8_t* codes,
+                                     uint8_t* scales) {
   if (!x || !codes || !scales) return 1;
   if (M < 0 || K <= 0 || K % MX_GROUP != 0) return 2;
   if (M == 0) return 0;
   float* y = (float*)malloc((size_t)M * (size_t)K * sizeof(float));
   if (!y) return 3;
-  int rc = bro_ref_rotate(x, M, K, ldx, block, y);
+  int rc = bro_ref_rotate_rs(x, M, K, ldx, block, signs, y);
   if (rc == 0) rc = bro_ref_quantize(y, M, K, codes, scales);
   free(y);
   return rc;
+}
+
+int bro_ref_rotate_quantize_mxfp4(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
+                                  int block, uint8_t* codes, uint8_t* scales) {
+  return bro_ref_rotate_quantize_mxfp4_rs(x, M, K, ldx, block, NULL, codes, scales);
 }
 
 int bro_ref_pack_weights(const uint16_t* w, int64_t N, int64_t K, int64_t ldw, int block,

@@ -56,6 +56,14 @@ float bro_ref_hadamard_norm(int64_t block);
 int bro_ref_rotate(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                    float* y);
 
+/* Randomised block rotation (Sec. 5.1: "block-wise randomized Hadamard rotations"; the random
+ * Hadamard construction of the rotation methods the paper builds on): R_i = diag(s) H / sqrt(block)
+ * with s a vector of +-1 over the K channels, so y[m, :] = (x[m, :] * s) R_block.  signs_bf16 holds
+ * one bf16 value per channel whose SIGN BIT is s (the magnitude is ignored); NULL means all +1.
+ * The random draw itself is an input: the oracle consumes no random numbers. */
+int bro_ref_rotate_rs(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                      const uint16_t* signs_bf16, float* y);
+
 /* MXFP4 quantisation of fp32 rows (Sec. 4.1): per group of 32, E8M0 scale + 32 E2M1 codes. */
 int bro_ref_quantize(const float* y, int64_t rows, int64_t K, uint8_t* codes, uint8_t* scales);
 
@@ -66,6 +74,11 @@ int bro_ref_decode(const uint8_t* codes, const uint8_t* scales, int64_t rows, in
 /* Activation path: rotate then quantise. */
 int bro_ref_rotate_quantize_mxfp4(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx,
                                   int block, uint8_t* codes, uint8_t* scales);
+
+/* Activation path with the randomised rotation (signs_bf16 as in bro_ref_rotate_rs). */
+int bro_ref_rotate_quantize_mxfp4_rs(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                                     int block, const uint16_t* signs_bf16, uint8_t* codes,
+                                     uint8_t* scales);
 
 /* Weight path: identical arithmetic applied to the rows of W[N, K] (offline). */
 int bro_ref_pack_weights(const uint16_t* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,

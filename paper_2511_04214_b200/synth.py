@@ -59,6 +59,14 @@ def weights(N: int, K: int, seed: int, std: float = 0.02) -> torch.Tensor:
     return w.to(torch.bfloat16)
 
 
+def rotation_signs(K: int, seed: int) -> torch.Tensor:
+    """bf16 [K] vector of +1 / -1, drawn uniformly: the diagonal of the randomised block rotation.
+    The draw is an input of the method on both sides (oracle and CUDA); neither draws its own."""
+    g = torch.Generator(device="cpu").manual_seed(int(seed) + 104729)
+    bits = torch.randint(0, 2, (K,), generator=g, dtype=torch.int32)
+    return (1.0 - 2.0 * bits.to(torch.float32)).to(torch.bfloat16)
+
+
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """View a CPU bf16 tensor as a numpy uint16 array of its bit patterns (no copy)."""
     assert t.dtype == torch.bfloat16 and t.device.type == "cpu"

@@ -179,3 +179,66 @@ def test_bad_arguments_rejected():
         oracle.rotate(x, 0)           # global needs a power-of-two K
     with pytest.raises(ValueError):
         oracle.rotate(x, 48)          # not a power of two
+
+
+# ---- randomised block rotation: R_i = diag(s) H / sqrt(B)  (Sec. 5.1) ---------------------------
+def sign_bits(rng, K):
+    s = np.where(rng.random(K) < 0.5, 1.0, -1.0).astype(np.float32)
+    return s, to_bits(s)
+
+
+@pytest.mark.parametrize("B", [32, 64, 128])
+def test_randomised_rotation_is_orthogonal_and_is_diag_s_times_hadamard(B):
+    rng = np.random.default_rng(B)
+    s, sb = sign_bits(rng, B)
+    R = oracle.rotate(to_bits(np.eye(B, dtype=np.float32)), B, sb).astype(np.float64)   # rows e_j R
+    tol = 0.0 if B == 64 else 1e-6
+    assert np.max(np.abs(R @ R.T - np.eye(B))) <= tol                                 # Eq. 1
+    expect = np.diag(s.astype(np.float64)) @ sylvester(B) / np.sqrt(B)
+    assert np.max(np.abs(R - expect)) <= 1e-7
+
+
+def test_randomised_rotation_equals_plain_rotation_of_sign_flipped_input():
+    """x diag(s) is exact in bf16, so rotating with signs must equal, bit for bit, the plain rotation
+    of an input that was negated channel by channel beforehand (done here in numpy)."""
+    rng = np.random.default_rng(5)
+    K = 256
+    x = synth.activations(9, K, seed=3).float().numpy()
+    s, sb = sign_bits(rng, K)
+    for B in (32, 128, 0):
+        a = oracle.rotate(to_bits(x), B, sb)
+        b = oracle.rotate(to_bits(x * s[None, :]), B)
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+    allplus = to_bits(np.ones(K, dtype=np.float32))
+    assert np.array_equal(oracle.rotate(to_bits(x), 32, allplus), oracle.rotate(to_bits(x), 32))
+    # only the sign bit of the sign vector counts
+    assert np.array_equal(oracle.rotate(to_bits(x), 32, to_bits(s * 3.0)), oracle.rotate(to_bits(x), 32, sb))
+
+
+def test_randomised_rotation_leaves_the_unquantised_product_unchanged():
+    """(x R)(W R)^T = x W^T for the same sign vector on both operands; with different sign vectors
+    it is not (a plausible mistake: signs applied to one side only)."""
+    rng = np.random.default_rng(8)
+    M, N, K = 5, 7, 128
+    x = small_int_rows(rng, M, K)
+    w = small_int_rows(rng, N, K)
+    s, sb = sign_bits(rng, K)
+    xr = oracle.rotate(to_bits(x), 32, sb).astype(np.float64)
+    wr = oracle.rotate(to_bits(w), 32, sb).astype(np.float64)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    assert np.max(np.abs(xr @ wr.T - ref)) <= 1e-4 * np.max(np.abs(ref))
+    w_plain = oracle.rotate(to_bits(w), 32).astype(np.float64)
+    assert np.max(np.abs(xr @ w_plain.T - ref)) > 1e-2 * np.max(np.abs(ref))
+
+
+def test_randomised_quantisation_uses_the_rotated_values():
+    x = synth.activations(6, 128, seed=12)
+    sb = synth.bf16_bits(synth.rotation_signs(128, seed=1))
+    y = oracle.rotate(synth.bf16_bits(x), 64, sb)
+    c1, s1 = oracle.quantize(y)
+    c2, s2 = oracle.rotate_quantize_mxfp4(synth.bf16_bits(x), 64, sb)
+    assert np.array_equal(c1, c2) and np.array_equal(s1, s2)
+    c3, _ = oracle.rotate_quantize_mxfp4(synth.bf16_bits(x), 64)
+    assert not np.array_equal(c1, c3)
+    c4, s4 = oracle.pack_weights(synth.bf16_bits(x), 64, sb)
+    assert np.array_equal(c4, c2) and np.array_equal(s4, s2)
