@@ -139,6 +139,25 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
                       int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Randomised block rotation (Sec. 5.1, "block-wise randomized Hadamard rotations"): the same three
+ * operations with R_i = diag(s) H_block / sqrt(block), s a vector of +-1 over the K channels, i.e.
+ * channel k of every row is multiplied by s_k (exactly, a sign-bit flip) before the transform.
+ *   signs_bf16  device, [K] bf16, 16-byte aligned; only the SIGN BIT of each value is used
+ *               (+1 / -1).  The caller draws it; the library consumes no random numbers.
+ * Activations and weights must use the same sign vector, so that (x R)(W R)^T = x W^T.
+ * All other arguments and requirements are those of the plain entry points.
+ */
+bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                                        int block, const void* signs_bf16, void* codes,
+                                        void* scales, bro_layout layout, void* stream);
+bro_status bro_pack_weights_rs(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                               const void* signs_bf16, void* wcodes, void* wscales, void* stream);
+bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                         const void* signs_bf16, const void* wcodes, const void* wscales, int64_t N,
+                         void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/*
  * bro_linear for a caller whose activations and result live in HOST memory (pinned memory gives
  * asynchronous copies).  Copies x_host[M, K] (dense, ldx = K) to the device staging buffer,
  * runs bro_linear, and copies y[M, N] (dense) back to y_host, all on `stream`.

@@ -25,6 +25,7 @@ EXPORTS = [
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host", "bro_linear_static",
+    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs",
 ]
 
 
@@ -68,6 +69,12 @@ def _load() -> ctypes.CDLL:
     L.bro_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p, sz, p]
     L.bro_linear_host.restype = ci
     L.bro_linear_host.argtypes = [p, i64, i64, ci, p, p, i64, p, p, p, p, sz, p]
+    L.bro_rotate_quantize_mxfp4_rs.restype = ci
+    L.bro_rotate_quantize_mxfp4_rs.argtypes = [p, i64, i64, i64, ci, p, p, p, ci, p]
+    L.bro_pack_weights_rs.restype = ci
+    L.bro_pack_weights_rs.argtypes = [p, i64, i64, i64, ci, p, p, p, p]
+    L.bro_linear_rs.restype = ci
+    L.bro_linear_rs.argtypes = [p, i64, i64, i64, ci, p, p, p, i64, p, i64, p, sz, p]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
     return L
@@ -202,3 +209,33 @@ def linear_static(x: torch.Tensor, block: int, wcodes, wscales, N: int, y: torch
     if code == 5:
         raise BroError(code, "bro_linear_static: " + lib.bro_last_cuda_error().decode())
     _check(code, "bro_linear_static")
+
+
+def _ld(t, n):
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), n)
+
+
+def rotate_quantize_mxfp4_rs(x: torch.Tensor, block: int, signs: torch.Tensor, codes, scales,
+                             layout: int = LAYOUT_GEMM, stream=None) -> None:
+    """Randomised rotation: ``signs`` is a bf16 [K] device vector of +1 / -1."""
+    assert x.dtype == torch.bfloat16 and signs.dtype == torch.bfloat16 and signs.numel() == x.shape[1]
+    M, K = x.shape
+    _check(lib.bro_rotate_quantize_mxfp4_rs(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), _ptr(codes),
+                                            _ptr(scales), layout, _stream(stream)),
+           "bro_rotate_quantize_mxfp4_rs")
+
+
+def pack_weights_rs(w: torch.Tensor, block: int, signs: torch.Tensor, wcodes, wscales, stream=None) -> None:
+    assert w.dtype == torch.bfloat16 and signs.dtype == torch.bfloat16 and signs.numel() == w.shape[1]
+    N, K = w.shape
+    _check(lib.bro_pack_weights_rs(_ptr(w), N, K, _ld(w, K), block, _ptr(signs), _ptr(wcodes),
+                                   _ptr(wscales), _stream(stream)), "bro_pack_weights_rs")
+
+
+def linear_rs(x: torch.Tensor, block: int, signs: torch.Tensor, wcodes, wscales, N: int, y: torch.Tensor,
+              workspace: torch.Tensor, stream=None) -> None:
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16 and signs.dtype == torch.bfloat16
+    M, K = x.shape
+    _check(lib.bro_linear_rs(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), _ptr(wcodes), _ptr(wscales), N,
+                             _ptr(y), _ld(y, N), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "bro_linear_rs")

@@ -125,7 +125,8 @@ namespace {
 
 // ---- rotate + quantise ---------------------------------------------------------------------------
 bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, int block,
-                                  void* codes, void* scales, bro_layout layout, cudaStream_t st) {
+                                  const void* signs, void* codes, void* scales, bro_layout layout,
+                                  cudaStream_t st) {
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (M == 0 && (layout == BRO_LAYOUT_CANONICAL || layout == BRO_LAYOUT_GEMM)) return BRO_OK;
@@ -135,14 +136,15 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
   if (K % B != 0) return BRO_ERR_SHAPE;
   if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
-  if (ldx % 8 != 0 || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16)) return BRO_ERR_ALIGN;
+  if (ldx % 8 != 0 || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(signs, 16))
+    return BRO_ERR_ALIGN;
   if (M == 0) return BRO_OK;
   DeviceInfo di;
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
 
   if (B > 128) {
-    return bro::rqg::launch(x, M, K, ldx, codes, scales, layout, gemm_scale_kblocks(K), di.sm_count, st);
+    return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, layout, gemm_scale_kblocks(K), di.sm_count, st);
   }
 
   CUtensorMap tmx;
@@ -159,13 +161,14 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   p.scales = static_cast<uint8_t*>(scales);
   p.scale_kblocks = gemm_scale_kblocks(K);
   p.layout = (int)layout;
+  p.signs = static_cast<const uint16_t*>(signs);
   const int64_t tiles = p.tiles_m * p.tiles_k;
   const int grid = (int)(tiles < di.sm_count ? tiles : di.sm_count);
 
   // (All three instantiations share one function-pointer type, so the opt-in to large dynamic
   // shared memory is keyed by the kernel's address, per device.)
   auto go = [&](void (*kernel)(CUtensorMap, Params), int which) -> bro_status {
-    static bool attr_done[64][3] = {};
+    static bool attr_done[64][6] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (!attr_done[dev][which]) {
@@ -178,10 +181,17 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
                ? BRO_OK
                : BRO_ERR_CUDA;
   };
+  if (signs) {
+    switch (B) {
+      case 32: return go(bro::rq::rotate_quantize_kernel<5, true>, 3);
+      case 64: return go(bro::rq::rotate_quantize_kernel<6, true>, 4);
+      default: return go(bro::rq::rotate_quantize_kernel<7, true>, 5);
+    }
+  }
   switch (B) {
-    case 32: return go(bro::rq::rotate_quantize_kernel<5>, 0);
-    case 64: return go(bro::rq::rotate_quantize_kernel<6>, 1);
-    default: return go(bro::rq::rotate_quantize_kernel<7>, 2);
+    case 32: return go(bro::rq::rotate_quantize_kernel<5, false>, 0);
+    case 64: return go(bro::rq::rotate_quantize_kernel<6, false>, 1);
+    default: return go(bro::rq::rotate_quantize_kernel<7, false>, 2);
   }
 }
 
@@ -250,13 +260,26 @@ bro_status bro_last_device_status(void* stream) {
 
 bro_status bro_rotate_quantize_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                      void* codes, void* scales, bro_layout layout, void* stream) {
-  return launch_rotate_quantize(x_bf16, M, K, ldx, block, codes, scales, layout,
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, nullptr, codes, scales, layout,
+                                static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                        const void* signs_bf16, void* codes, void* scales, bro_layout layout,
+                                        void* stream) {
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, signs_bf16, codes, scales, layout,
+                                static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_pack_weights_rs(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                               const void* signs_bf16, void* wcodes, void* wscales, void* stream) {
+  return launch_rotate_quantize(w_bf16, N, K, ldw, block, signs_bf16, wcodes, wscales, BRO_LAYOUT_GEMM,
                                 static_cast<cudaStream_t>(stream));
 }
 
 bro_status bro_pack_weights(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
                             void* wcodes, void* wscales, void* stream) {
-  return launch_rotate_quantize(w_bf16, N, K, ldw, block, wcodes, wscales, BRO_LAYOUT_GEMM,
+  return launch_rotate_quantize(w_bf16, N, K, ldw, block, nullptr, wcodes, wscales, BRO_LAYOUT_GEMM,
                                 static_cast<cudaStream_t>(stream));
 }
 
@@ -290,9 +313,9 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
                            workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream));
 }
 
-bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,
-                      const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
-                      size_t workspace_bytes, void* stream) {
+static bro_status linear_impl(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs,
+                              const void* wcodes, const void* wscales, int64_t N, void* y_bf16, int64_t ldy,
+                              void* workspace, size_t workspace_bytes, void* stream) {
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
   if (M == 0 || N == 0) return BRO_OK;
   if (!x_bf16 || !wcodes || !wscales || !y_bf16 || !workspace) return BRO_ERR_NULL;
@@ -302,10 +325,26 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
   uint8_t* acodes = ws;
   uint8_t* ascales = acodes + align_up(bro_codes_bytes(M, K), 1024);
   uint8_t* gws = ascales + align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 1024);
-  bro_status rc = bro_rotate_quantize_mxfp4(x_bf16, M, K, ldx, block, acodes, ascales, BRO_LAYOUT_GEMM, stream);
+  bro_status rc = launch_rotate_quantize(x_bf16, M, K, ldx, block, signs, acodes, ascales, BRO_LAYOUT_GEMM,
+                                         static_cast<cudaStream_t>(stream));
   if (rc != BRO_OK) return rc;
   return bro_gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
                         bro_gemm_workspace_bytes(M, N, K), stream);
+}
+
+bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,
+                      const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  return linear_impl(x_bf16, M, K, ldx, block, nullptr, wcodes, wscales, N, y_bf16, ldy, workspace,
+                     workspace_bytes, stream);
+}
+
+bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs_bf16,
+                         const void* wcodes, const void* wscales, int64_t N, void* y_bf16, int64_t ldy,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+  if (!signs_bf16) return BRO_ERR_NULL;
+  return linear_impl(x_bf16, M, K, ldx, block, signs_bf16, wcodes, wscales, N, y_bf16, ldy, workspace,
+                     workspace_bytes, stream);
 }
 
 bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block, const void* wcodes,

@@ -42,7 +42,18 @@ struct Params {
   uint8_t* scales;
   int64_t scale_kblocks;        // GEMM layout: 512-byte blocks per 128-row block
   int layout;                   // bro_layout
+  const uint16_t* signs;        // [K] bf16 +-1 (randomised rotation, kernels with SIGNS) or nullptr
 };
+
+// x diag(s): flip the bf16 sign bits of a 16-byte chunk of x where the sign vector is negative.
+// One three-input logic operation per 32-bit word (x ^ (s & 0x80008000)); exact.
+__device__ __forceinline__ uint4 apply_signs(uint4 q, uint4 sg) {
+  q.x ^= sg.x & 0x80008000u;
+  q.y ^= sg.y & 0x80008000u;
+  q.z ^= sg.z & 0x80008000u;
+  q.w ^= sg.w & 0x80008000u;
+  return q;
+}
 
 __device__ __forceinline__ uint32_t pack_e2m1x8(float r0, float r1, float r2, float r3, float r4,
                                                 float r5, float r6, float r7) {
@@ -168,7 +179,9 @@ __device__ __forceinline__ uint32_t quantize_group(const uint64_t (&P)[16], uint
   return s;
 }
 
-template <int LOG2B>
+// SIGNS: the randomised rotation R_i = diag(s) H / sqrt(block) (paper Sec. 5.1) — the channel signs
+// are applied to the bf16 inputs as they leave shared memory; everything else is unchanged.
+template <int LOG2B, bool SIGNS>
 __global__ void __launch_bounds__(kThreads, 1)
 rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -247,9 +260,16 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
       if (!mbar_wait(bar_base + 8 * stage, phase, SITE_RQ_FULL)) break;
       const uint32_t src = smem_base + stage * kStageBytes + row_off;
       uint64_t P[16];
+      uint4 sg[4] = {};
+      if (SIGNS && (tk * (kTileCols / 32) + g) * 32 < (int)p.K) {
+        const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (tk * kTileCols + g * 32));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sg[j] = __ldg(sp + j);
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint4 q = lds128(src + ((((uint32_t)gg * 4u + j) ^ sw) << 4));
+        uint4 q = lds128(src + ((((uint32_t)gg * 4u + j) ^ sw) << 4));
+        if (SIGNS) q = apply_signs(q, sg[j]);
         unpack_stage1(q, P + 4 * j);
       }
       __syncwarp();

@@ -26,6 +26,7 @@ struct Params {
   int log2k;
   int threads_per_row;   // K / 32
   int rows_per_iter;     // blockDim.x / threads_per_row
+  const uint16_t* signs; // [K] bf16 +-1 for the randomised rotation diag(s) H / sqrt(K), or nullptr
 };
 
 template <int kMaxThreads>
@@ -39,6 +40,13 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   const int64_t row_iters = (p.M + p.rows_per_iter - 1) / p.rows_per_iter;
   griddep_launch_dependents();
   griddep_wait();               // x may be written, codes/scales still read, by the kernel before
+  // a thread always works on the same 32 channels, so its slice of the sign vector is loaded once
+  uint4 sg[4] = {};
+  if (p.signs) {
+    const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)gi * 32);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sg[j] = __ldg(sp + j);
+  }
 
   for (int64_t it = blockIdx.x; it < row_iters; it += gridDim.x) {
     const int64_t row = it * p.rows_per_iter + rs;
@@ -49,7 +57,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint4 q = live ? __ldg(src + j) : make_uint4(0u, 0u, 0u, 0u);
-        rq::unpack_stage1(q, P + 4 * j);
+        rq::unpack_stage1(rq::apply_signs(q, sg[j]), P + 4 * j);
       }
     }
     rq::fwht32_stages_2_to_16(P);
@@ -99,8 +107,8 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   }
 }
 
-inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, void* codes, void* scales,
-                         bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
+                         void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M;
@@ -110,6 +118,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, void*
   p.scales = static_cast<uint8_t*>(scales);
   p.scale_kblocks = scale_kblocks;
   p.layout = (int)layout;
+  p.signs = static_cast<const uint16_t*>(signs);
   int lg = 0;
   while (((int64_t)1 << lg) < K) ++lg;
   p.log2k = lg;
