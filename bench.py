@@ -447,12 +447,20 @@ def run_rotate_quantize_only(args):
     t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
     torch.cuda._sleep(int(2e7))
     t_all0.record()
+    # One step = one launch per rotation size.  Per-size times come from CUDA events around groups
+    # of `group` back-to-back launches of that size (cycling through the ring of inputs, so every
+    # launch reads its 134 MB from HBM); an event pair around every single launch would add its own
+    # latency to a 30 us kernel.
+    group = 2 * ring
+    n_groups = max(1, steps // group)
+    steps = n_groups * group
     evs = {b: [] for b in blocks}
-    for i in range(steps):
+    for gi in range(n_groups):
         for b in blocks:
             a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+            for i in range(group):
+                bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
             c.record()
             evs[b].append((a, c))
     t_all1.record()
@@ -461,7 +469,7 @@ def run_rotate_quantize_only(args):
     assert bro.last_device_status() == 0
     bytes_per_launch = M * K * 2.53125
     for b in blocks:
-        ts = [a.elapsed_time(c) for a, c in evs[b]]
+        ts = [a.elapsed_time(c) / group for a, c in evs[b]]
         per_block[str(b if b else K)] = {"us": statistics.mean(ts) * 1e3, "gbs": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9,
                                          "frac_of_measured_copy": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     ms_total = t_all0.elapsed_time(t_all1)
@@ -475,7 +483,8 @@ def run_rotate_quantize_only(args):
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                        "traffic": None, "algorithmic_bytes": bytes_per_launch}}
+                        "traffic": None, "algorithmic_bytes": bytes_per_launch,
+                        "timing": f"CUDA events around groups of {group} back-to-back launches, {n_groups} groups per size"}}
     print(json.dumps(out), flush=True)
 
 

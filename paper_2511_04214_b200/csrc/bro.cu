@@ -9,6 +9,7 @@
 #include "bro_common.cuh"
 #include "rotate_quantize.cuh"
 #include "rotate_quantize_global.cuh"
+#include "rotate_quantize_direct.cuh"
 #include "gemm_mxfp4.cuh"
 #include "gemm_mxfp4_2cta.cuh"
 
@@ -146,6 +147,16 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   if (B > 128) {
     return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, layout, gemm_scale_kblocks(K), di.sm_count, st);
   }
+
+  // Register-streaming kernel by default; BRO_RQ_TMA=1 selects the TMA-ring kernel (also used when
+  // the task index would not fit 31 bits).
+  // (it wins for block 32 at every size and for small inputs; for blocks of 64 / 128 on large
+  // inputs its extra registers cost occupancy and the TMA ring is faster)
+  bool direct = bro::rqd::supports(M, K, layout, gemm_scale_kblocks(K)) && (B == 32 || M * K <= ((int64_t)1 << 23));
+  if (const char* e = getenv("BRO_RQ_TMA")) direct = direct && atoi(e) == 0;
+  if (direct)
+    return bro::rqd::launch(x, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs, codes, scales, layout,
+                            gemm_scale_kblocks(K), di.sm_count, st);
 
   CUtensorMap tmx;
   rc = make_map_2d(&tmx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, (uint64_t)K, (uint64_t)M,

@@ -1,0 +1,176 @@
+// Kernel 1 (register-streaming form): fused block-Hadamard rotation + MXFP4 quantisation
+// (paper Sec. 4.3 Eq. 1, Sec. 4.1) without a shared-memory stage.
+//
+// Same arithmetic contract as rotate_quantize.cuh (whose helpers it reuses): a thread owns one MX
+// group of 32 consecutive channels, butterflies with ascending stride in fp32, one multiply by
+// fp32(1/sqrt(block)), amax -> E8M0 exponent, round-to-nearest-even E2M1 codes.
+//
+// What differs is how the bytes travel.  The 32 lanes of a warp take 32 consecutive groups of one
+// row (2 KiB of contiguous bf16), each lane loading its 64 bytes with four 16-byte loads straight
+// into registers, and the loads of the warp's NEXT task are issued before the current one is
+// computed.  Nothing goes through shared memory: in the TMA-ring form the shared-memory port carries
+// every byte twice (TMA write, then the consumers' loads) and all consumer warps wake on the same
+// barrier, which together cost about a third of its run time on a [16384, 4096] tensor; here more
+// warps are resident and they drift apart, so loads, arithmetic and stores of different warps
+// overlap.  Blocks of 64 / 128 channels pair lanes l ^ 1 (and l ^ 2) for their last one / two stages.
+#pragma once
+
+#include "bro_common.cuh"
+#include "rotate_quantize.cuh"
+
+namespace bro {
+namespace rqd {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+struct Params {
+  const uint16_t* x;
+  int64_t M, K, ldx;
+  uint8_t* codes;               // [M, K/2]
+  uint8_t* scales;
+  int64_t scale_kblocks;        // tensor-core layout: 512-byte blocks per 128-row block
+  int layout;                   // bro_layout
+  const uint16_t* signs;        // [K] bf16 +-1 (kernels with SIGNS) or nullptr
+  int rows_padded;              // rows the task grid covers (a multiple of 128 for the tensor-core layout)
+  int groups_padded;            // groups per row it covers (scale padding included)
+  int chunks_per_row;           // ceil(groups_padded / 32)
+  int total_tasks;              // rows_padded * chunks_per_row; one task = one warp, 32 groups of a row
+};
+
+template <int LOG2B, bool SIGNS>
+__global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(const Params p) {
+  const int lane = threadIdx.x & 31;
+  const int num_warps = (int)gridDim.x * kWarps;
+  const int ng = (int)(p.K >> 5);
+  constexpr uint32_t cbits = rq::norm_bits<LOG2B>();
+
+  griddep_launch_dependents();
+  griddep_wait();               // x may be written, codes/scales still read, by the kernel before
+
+  // task -> (row, chunk); advanced incrementally (no division in the loop)
+  int task = (int)blockIdx.x * kWarps + (int)(threadIdx.x >> 5);
+  int row = task / p.chunks_per_row, chunk = task - row * p.chunks_per_row;
+  const int step_row = num_warps / p.chunks_per_row, step_chunk = num_warps - step_row * p.chunks_per_row;
+
+  auto load = [&](int r, int c, uint4 (&q)[4]) {
+    const int g = c * 32 + lane;
+    if (r < p.M && g < ng) {
+      const uint4* src = reinterpret_cast<const uint4*>(p.x + (int64_t)r * p.ldx + (int64_t)g * 32);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) q[j] = __ldg(src + j);
+      if (SIGNS) {
+        const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)g * 32);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q[j] = rq::apply_signs(q[j], __ldg(sp + j));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) q[j] = make_uint4(0u, 0u, 0u, 0u);   // padding quantises to zeros
+    }
+  };
+
+  uint4 cur[4], nxt[4];
+  if (task < p.total_tasks) load(row, chunk, cur);
+  while (task < p.total_tasks) {
+    // the next task of this warp: issue its loads now, use them in the next iteration
+    const int ntask = task + num_warps;
+    int nrow = row + step_row, nchunk = chunk + step_chunk;
+    if (nchunk >= p.chunks_per_row) { nchunk -= p.chunks_per_row; ++nrow; }
+    if (ntask < p.total_tasks) load(nrow, nchunk, nxt);
+
+    uint64_t P[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rq::unpack_stage1(cur[j], P + 4 * j);
+    rq::fwht32_stages_2_to_16(P);
+    if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
+    if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
+    uint32_t w[4];
+    const uint32_t s = rq::quantize_group(P, cbits, w);
+
+    const int g = chunk * 32 + lane;
+    const bool live = row < p.M && g < ng;
+    if (live)
+      *reinterpret_cast<uint4*>(p.codes + (int64_t)row * (p.K >> 1) + (int64_t)g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    // scale bytes of 4 consecutive groups -> one 32-bit word in the lane with g % 4 == 0
+    uint32_t sb = live ? s : 0u;
+    sb |= __shfl_xor_sync(0xFFFFFFFFu, sb, 1) << 8;
+    sb |= __shfl_xor_sync(0xFFFFFFFFu, sb, 2) << 16;
+    if ((lane & 3) == 0 && g < p.groups_padded) {
+      if (p.layout == BRO_LAYOUT_GEMM) {
+        // 512-byte block (row / 128, g / 4): byte (r % 32) * 16 + ((r % 128) / 32) * 4 + g % 4
+        const int64_t off = ((int64_t)(row >> 7) * p.scale_kblocks + (g >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
+        *reinterpret_cast<uint32_t*>(p.scales + off) = sb;
+      } else if (row < p.M) {
+        uint8_t* dst = p.scales + (int64_t)row * ng + g;
+        if (g + 4 <= ng && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+          *reinterpret_cast<uint32_t*>(dst) = sb;
+        } else {
+          for (int i = 0; i < 4 && g + i < ng; ++i) dst[i] = (uint8_t)(sb >> (8 * i));
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+    task = ntask;
+    row = nrow;
+    chunk = nchunk;
+  }
+}
+
+// Rows x padded groups must fit 31 bits of task index; larger problems use the TMA-ring kernel.
+inline bool supports(int64_t M, int64_t K, bro_layout layout, int64_t scale_kblocks) {
+  const int64_t rows = layout == BRO_LAYOUT_GEMM ? (M + 127) / 128 * 128 : M;
+  const int64_t groups = layout == BRO_LAYOUT_GEMM ? scale_kblocks * 4 : K / 32;
+  return rows * ((groups + 31) / 32) < ((int64_t)1 << 30);
+}
+
+template <int LOG2B, bool SIGNS>
+inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
+  auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS>;
+  static int blocks_per_sm[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (blocks_per_sm[dev] == 0) {
+    int n = 0;
+    if (!cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0), "occupancy(rotate_quantize_direct)"))
+      return BRO_ERR_CUDA;
+    blocks_per_sm[dev] = n > 0 ? n : 1;
+  }
+  const int64_t want = ((int64_t)p.total_tasks + kWarps - 1) / kWarps;
+  const int64_t cap = (int64_t)sm_count * blocks_per_sm[dev];
+  const unsigned grid = (unsigned)(want < cap ? want : cap);
+  return cuda_ok(launch_kernel(kernel, grid, kThreads, 0, st, 1, p), "rotate_quantize_direct launch") ? BRO_OK
+                                                                                                       : BRO_ERR_CUDA;
+}
+
+inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs, void* codes,
+                         void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+  Params p;
+  p.x = static_cast<const uint16_t*>(x);
+  p.M = M; p.K = K; p.ldx = ldx;
+  p.codes = static_cast<uint8_t*>(codes);
+  p.scales = static_cast<uint8_t*>(scales);
+  p.scale_kblocks = scale_kblocks;
+  p.layout = (int)layout;
+  p.signs = static_cast<const uint16_t*>(signs);
+  p.rows_padded = (int)(layout == BRO_LAYOUT_GEMM ? (M + 127) / 128 * 128 : M);
+  p.groups_padded = (int)(layout == BRO_LAYOUT_GEMM ? scale_kblocks * 4 : K / 32);
+  p.chunks_per_row = (p.groups_padded + 31) / 32;
+  p.total_tasks = p.rows_padded * p.chunks_per_row;
+  if (signs) {
+    switch (log2b) {
+      case 5: return launch_one<5, true>(p, sm_count, st);
+      case 6: return launch_one<6, true>(p, sm_count, st);
+      default: return launch_one<7, true>(p, sm_count, st);
+    }
+  }
+  switch (log2b) {
+    case 5: return launch_one<5, false>(p, sm_count, st);
+    case 6: return launch_one<6, false>(p, sm_count, st);
+    default: return launch_one<7, false>(p, sm_count, st);
+  }
+}
+
+}  // namespace rqd
+}  // namespace bro
