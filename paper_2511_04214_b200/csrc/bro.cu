@@ -107,10 +107,11 @@ bro_status bro::gemm::make_codes_map(CUtensorMap* map, const void* base, int64_t
                      (uint64_t)(K / 2), 128, (uint32_t)box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-// bf16 output [M, ldy]: box = 32 columns (64 bytes) x 128 rows, 64-byte swizzle (epilogue staging).
+// bf16 output [M, ldy]: box = 64 columns (128 bytes) x 32 rows (what one epilogue warp stores at a
+// time), 128-byte swizzle to match its staging buffer.
 bro_status bro::gemm::make_out_map(CUtensorMap* map, const void* y, int64_t M, int64_t N, int64_t ldy) {
   return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy * 2,
-                     bro::gemm::kChunkCols, bro::gemm::kBM, CU_TENSOR_MAP_SWIZZLE_64B);
+                     2 * bro::gemm::kChunkCols, 32, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // Scale tensor in the tensor-core layout viewed as 32-bit words: one row per 128-row block

@@ -14,10 +14,10 @@
 //               (tcgen05.cp) and issues four tcgen05.mma kind::mxf4.block_scale (K = 64 each)
 //               per K step into one of two fp32 accumulators in TMEM; tcgen05.commit releases the
 //               shared-memory stage and, after the last K step, hands the accumulator over.
-//   warps 2..5  epilogue: tcgen05.ld the accumulator in 32-column chunks (one TMEM lane quadrant
-//               per warp), convert to bf16, stage the chunk in shared memory (64-byte swizzle)
-//               and write it with a TMA store (which also clips the ragged edges); the fp32
-//               output mode stores straight from registers.
+//   warps 2..5  epilogue, each warp on its own for the 32 rows of its TMEM lane quadrant:
+//               tcgen05.ld of 64 columns (the next 64 in flight), convert to bf16, stage in the
+//               warp's shared-memory buffer (128-byte swizzle), one TMA store of a 64 x 32 box
+//               (which also clips the ragged edges); the fp32 output mode stores from registers.
 // TMEM holds 512 columns.  For BN = 256 two full accumulators plus the scale columns do not
 // fit, so the two accumulators overlap by 32 columns ([0,256) and [224,480)): the epilogue drains
 // the shared 32 columns first and releases them early, and the next tile's MMAs start as soon as
@@ -191,6 +191,23 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src,
                "r"(src), "r"(x), "r"(y)
                : "memory");
 }
+// One-lane forms for a converged warp (`issue` non-zero in the issuing lane; operands uniform).
+__device__ __forceinline__ void tma_store_2d_if(uint32_t issue, const CUtensorMap* m, uint32_t src, int x, int y) {
+  asm volatile(
+      "{ .reg .pred q; setp.ne.b32 q, %4, 0;\n\t"
+      "@q cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1]; }" ::"l"(
+          reinterpret_cast<uint64_t>(m)),
+      "r"(src), "r"(x), "r"(y), "r"(issue)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit_if(uint32_t issue) {
+  asm volatile("{ .reg .pred q; setp.ne.b32 q, %0, 0;\n\t@q cp.async.bulk.commit_group; }" ::"r"(issue) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read_if(uint32_t issue) {
+  asm volatile("{ .reg .pred q; setp.ne.b32 q, %0, 0;\n\t@q cp.async.bulk.wait_group.read %1; }" ::"r"(issue), "n"(N)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {
@@ -282,6 +299,108 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
       phase = next_phase;
     }
     tc_commit<CG>(issue, r.bar_acc_full + 8 * buf);    // accumulator complete (or abandoned) -> epilogue
+  }
+}
+
+// One epilogue warp's share of one finished accumulator: the 32 rows of its TMEM lane quadrant,
+// CHUNKS chunks of 32 columns, handled two chunks (64 columns) at a time.  The warp works on its
+// own — no barrier between warps: tcgen05.ld of the next pair is in flight while the current one is
+// converted to bf16, written to the warp's staging buffer (32 rows x 128 bytes, 128-byte swizzle)
+// and sent off with ONE TMA store of a 64 x 32 box, which clips rows beyond M and columns beyond N.
+// (Tried and slower: st.global straight from registers, and a transpose through shared memory
+// followed by coalesced 16-byte st.global — both make the whole kernel 15-20 % slower on
+// output-heavy shapes; the asynchronous TMA store is what keeps the epilogue off the critical path.)
+// Pair order: the pair that holds the columns shared with the other accumulator first (buffer 0
+// shares its last chunk, buffer 1 its first); `release_shared` / `release_all` are called once
+// those columns / all columns have been read into registers.
+template <int CHUNKS, bool OVERLAP, bool OUT_F32, typename ReleaseShared, typename ReleaseAll>
+__device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int lane, int row0, int n0, int64_t M,
+                                              int64_t N, void* y, int64_t ldy, const CUtensorMap* tmy,
+                                              uint32_t stage_buf, ReleaseShared release_shared,
+                                              ReleaseAll release_all) {
+  static_assert(CHUNKS % 2 == 0, "chunks are processed in pairs");
+  constexpr int PAIRS = CHUNKS / 2;
+  const int64_t row = (int64_t)row0 + lane;
+  const uint32_t issue = lane == 0 ? 1u : 0u;
+  auto pair_of = [&](int pi) { return (OVERLAP && buf == 0) ? (pi == 0 ? PAIRS - 1 : pi - 1) : pi; };
+  auto released = [&](int pi) {
+    if (pi == 0 || pi == PAIRS - 1) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (pi == 0) release_shared();
+        if (pi == PAIRS - 1) release_all();
+      }
+    }
+  };
+  auto store_f32 = [&](const uint32_t (&r)[32], int col0) {
+    if (row < M && col0 < N) {
+      float* dst = static_cast<float*>(y) + row * ldy + col0;
+      if ((int64_t)col0 + 32 <= N) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          reinterpret_cast<uint4*>(dst)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      } else {
+        for (int j = 0; j < 32 && col0 + j < N; ++j) dst[j] = __uint_as_float(r[j]);
+      }
+    }
+  };
+  auto emit = [&](const uint32_t (&r0)[32], const uint32_t (&r1)[32], int pr) {
+    const int col0 = n0 + pr * 2 * kChunkCols;
+    if (OUT_F32) {
+      store_f32(r0, col0);
+      store_f32(r1, col0 + kChunkCols);
+    } else {
+      uint32_t h[32];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r0[2 * j + 1])), "f"(__uint_as_float(r0[2 * j])));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[16 + j]) : "f"(__uint_as_float(r1[2 * j + 1])), "f"(__uint_as_float(r1[2 * j])));
+      }
+      // the TMA store that last read the staging buffer must be done reading it
+      bulk_wait_read_if<0>(issue);
+      __syncwarp();
+      // row `lane` of the box: 128 bytes, 16-byte pieces XOR-swizzled with lane & 7
+      const uint32_t rowaddr = stage_buf + (uint32_t)lane * 128u;
+      const uint32_t sw = (uint32_t)lane & 7u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) sts128(rowaddr + ((j ^ sw) << 4), h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+      fence_proxy_async_smem();
+      __syncwarp();
+      // A TMA store clips at 16-byte granularity: when N is not a multiple of 8 the ragged last
+      // pair is written from registers instead, element by element.
+      const bool ragged = ((N & 7) != 0) && ((int64_t)col0 + 2 * kChunkCols > N);
+      tma_store_2d_if((col0 < N && row0 < M && !ragged) ? issue : 0u, tmy, stage_buf, col0, row0);
+      bulk_commit_if(issue);           // (possibly empty) keeps the group count in step
+      if (ragged && row < M) {
+        uint16_t* dst = static_cast<uint16_t*>(y) + row * ldy + col0;
+#pragma unroll
+        for (int j = 0; j < 64; ++j)
+          if ((int64_t)col0 + j < N) dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
+      }
+    }
+  };
+  uint32_t ra[32], rb[32], rc[32], rd[32];
+  tc_ld32(tmem_acc + pair_of(0) * 2 * kChunkCols, ra);
+  tc_ld32(tmem_acc + pair_of(0) * 2 * kChunkCols + kChunkCols, rb);
+#pragma unroll
+  for (int pi = 0; pi < PAIRS; pi += 2) {
+    tc_wait_ld();
+    if (pi + 1 < PAIRS) {
+      tc_ld32(tmem_acc + pair_of(pi + 1) * 2 * kChunkCols, rc);
+      tc_ld32(tmem_acc + pair_of(pi + 1) * 2 * kChunkCols + kChunkCols, rd);
+    }
+    released(pi);
+    emit(ra, rb, pair_of(pi));
+    if (pi + 1 < PAIRS) {
+      tc_wait_ld();
+      if (pi + 2 < PAIRS) {
+        tc_ld32(tmem_acc + pair_of(pi + 2) * 2 * kChunkCols, ra);
+        tc_ld32(tmem_acc + pair_of(pi + 2) * 2 * kChunkCols + kChunkCols, rb);
+      }
+      released(pi + 1);
+      emit(rc, rd, pair_of(pi + 1));
+    }
   }
 }
 
@@ -384,81 +503,20 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
-    const int ep_tid = threadIdx.x - 64;    // 0..127
-    const int r_in_tile = q * 32 + lane;
-    uint32_t chunk_counter = 0;             // staging buffer = chunk_counter & 1
     int it = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++it) {
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++it) {
       const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
-      const int m0 = tm * kBM, n0 = tn * BN;
       const int buf = it & 1;
-      ok = named_barrier_and(2, 128, mbar_wait(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL));
-      if (!ok) break;
+      if (!mbar_wait_warp(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL)) break;
       tc_fence_after();
-      const uint32_t tmem_acc = tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16);
-      const int64_t row = (int64_t)m0 + r_in_tile;
-#pragma unroll 1
-      for (int ci = 0; ci < C::kChunks; ++ci) {
-        // Chunk order: the columns shared with the other accumulator first.  Buffer 0 shares its
-        // last chunk, buffer 1 its first.
-        const int c = (C::kOverlap && buf == 0) ? (ci == 0 ? C::kChunks - 1 : ci - 1) : ci;
-        uint32_t r[32];
-        tc_ld32(tmem_acc + c * kChunkCols, r);
-        tc_wait_ld();
-        if (ci == 0 || ci == C::kChunks - 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            if (ci == 0) mbar_arrive(bar_ovl_free + 8 * buf);
-            if (ci == C::kChunks - 1) mbar_arrive(bar_acc_free + 8 * buf);
-          }
-        }
-        const int col0 = n0 + c * kChunkCols;
-        if (OUT_F32) {
-          if (row < p.M && col0 < p.N) {
-            float* dst = static_cast<float*>(p.y) + row * p.ldy + col0;
-            if ((int64_t)col0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                reinterpret_cast<uint4*>(dst)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-            } else {
-              for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __uint_as_float(r[j]);
-            }
-          }
-        } else {
-          uint32_t h[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r[2 * j + 1])), "f"(__uint_as_float(r[2 * j])));
-          const uint32_t sbuf = sOut + (chunk_counter & 1u) * kStageOutBytes;
-          // the TMA store that last read this staging buffer (two chunks ago) must be done reading
-          if (ep_tid == 0) bulk_wait_read<1>();
-          named_barrier_sync(1, 128);
-          // row r of the chunk: 64 bytes at r*64, 16-byte pieces XOR-swizzled with (r >> 1) & 3
-          const uint32_t rowaddr = sbuf + (uint32_t)r_in_tile * 64u;
-          const uint32_t sw = ((uint32_t)r_in_tile >> 1) & 3u;
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            sts128(rowaddr + ((j ^ sw) << 4), h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-          fence_proxy_async_smem();
-          named_barrier_sync(1, 128);
-          // A TMA store clips at 16-byte granularity: when N is not a multiple of 8 the ragged last
-          // chunk is written from registers instead, element by element.
-          const bool ragged = ((p.N & 7) != 0) && ((int64_t)col0 + kChunkCols > p.N);
-          if (ep_tid == 0 && col0 < p.N && !ragged) tma_store_2d(&tmy, sbuf, col0, m0);
-          if (ep_tid == 0) bulk_commit();     // (possibly empty) keeps the group count in step
-          if (ragged && row < p.M) {
-            uint16_t* dst = static_cast<uint16_t*>(p.y) + row * p.ldy + col0;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if ((int64_t)col0 + j < p.N) dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
-          }
-          ++chunk_counter;
-        }
-      }
+      epilogue_tile<C::kChunks, C::kOverlap, OUT_F32>(
+          tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16), buf, lane, tm * kBM + q * 32, tn * BN, p.M, p.N,
+          p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u),
+          [&] { mbar_arrive(bar_ovl_free + 8 * buf); }, [&] { mbar_arrive(bar_acc_free + 8 * buf); });
     }
-    if (!OUT_F32 && ep_tid == 0) bulk_wait_all();
+    // the staging buffer must have been read before this CTA's shared memory goes away; the writes
+    // themselves complete with the kernel
+    if (!OUT_F32 && lane == 0) bulk_wait_read<0>();
   }
   tc_fence_before();
   __syncthreads();

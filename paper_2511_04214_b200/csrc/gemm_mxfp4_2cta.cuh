@@ -211,81 +211,23 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
   } else {
     // ------------------------------ epilogue (both CTAs) ------------------------------
     const int q = warp & 3;
-    const int ep_tid = threadIdx.x - 64;
-    const int r_in_tile = q * 32 + lane;
-    uint32_t chunk_counter = 0;
     int it = 0;
-    bool ok = true;
-    for (int tile = pair; tile < p.total_tiles && ok; tile += num_pairs, ++it) {
+    for (int tile = pair; tile < p.total_tiles; tile += num_pairs, ++it) {
       int tm, tn;
       tile_coords(tile, p, tm, tn);
-      const int m0 = tm * 256 + (int)rank * kBM;
-      const int n0 = tn * kBN;
       const int buf = it & 1;
-      ok = gemm::named_barrier_and(2, 128, mbar_wait(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL));
-      if (!ok) break;
+      if (!mbar_wait_warp(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL)) break;
       gemm::tc_fence_after();
-      const uint32_t tmem_acc = tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16);
-      const int64_t row = (int64_t)m0 + r_in_tile;
       const uint32_t ovl_free_leader = map_to_cta(bar_ovl_free + 8 * buf, 0);
       const uint32_t acc_free_leader = map_to_cta(bar_acc_free + 8 * buf, 0);
-#pragma unroll 1
-      for (int ci = 0; ci < kChunks; ++ci) {
-        // the columns shared with the other accumulator first: buffer 0 shares its last chunk,
-        // buffer 1 its first
-        const int c = (buf == 0) ? (ci == 0 ? kChunks - 1 : ci - 1) : ci;
-        uint32_t r[32];
-        gemm::tc_ld32(tmem_acc + c * kChunkCols, r);
-        gemm::tc_wait_ld();
-        if (ci == 0 || ci == kChunks - 1) {
-          gemm::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            if (ci == 0) mbar_arrive_cluster(ovl_free_leader);
-            if (ci == kChunks - 1) mbar_arrive_cluster(acc_free_leader);
-          }
-        }
-        const int col0 = n0 + c * kChunkCols;
-        if (OUT_F32) {
-          if (row < p.M && col0 < p.N) {
-            float* dst = static_cast<float*>(p.y) + row * p.ldy + col0;
-            if ((int64_t)col0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                reinterpret_cast<uint4*>(dst)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-            } else {
-              for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __uint_as_float(r[j]);
-            }
-          }
-        } else {
-          uint32_t h[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r[2 * j + 1])), "f"(__uint_as_float(r[2 * j])));
-          const uint32_t sbuf = sOut + (chunk_counter & 1u) * kStageOutBytes;
-          if (ep_tid == 0) gemm::bulk_wait_read<1>();
-          gemm::named_barrier_sync(1, 128);
-          const uint32_t rowaddr = sbuf + (uint32_t)r_in_tile * 64u;
-          const uint32_t sw = ((uint32_t)r_in_tile >> 1) & 3u;
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            gemm::sts128(rowaddr + ((j ^ sw) << 4), h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-          fence_proxy_async_smem();
-          gemm::named_barrier_sync(1, 128);
-          const bool ragged = ((p.N & 7) != 0) && ((int64_t)col0 + kChunkCols > p.N);
-          if (ep_tid == 0 && col0 < p.N && m0 < p.M && !ragged) gemm::tma_store_2d(&tmy, sbuf, col0, m0);
-          if (ep_tid == 0) gemm::bulk_commit();
-          if (ragged && row < p.M) {
-            uint16_t* dst = static_cast<uint16_t*>(p.y) + row * p.ldy + col0;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if ((int64_t)col0 + j < p.N) dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
-          }
-          ++chunk_counter;
-        }
-      }
+      gemm::epilogue_tile<kChunks, true, OUT_F32>(
+          tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16), buf, lane, tm * 256 + (int)rank * kBM + q * 32,
+          tn * kBN, p.M, p.N, p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u),
+          [&] { mbar_arrive_cluster(ovl_free_leader); }, [&] { mbar_arrive_cluster(acc_free_leader); });
     }
-    if (!OUT_F32 && ep_tid == 0) gemm::bulk_wait_all();
+    // the staging buffer must have been read before this CTA's shared memory goes away; the writes
+    // themselves complete with the kernel
+    if (!OUT_F32 && lane == 0) gemm::bulk_wait_read<0>();
   }
   gemm::tc_fence_before();
   __syncthreads();
