@@ -295,10 +295,9 @@ bro_status bro_pack_weights(const void* w_bf16, int64_t N, int64_t K, int64_t ld
                                 static_cast<cudaStream_t>(stream));
 }
 
-bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* wcodes,
-                          const void* wscales, int64_t M, int64_t N, int64_t K, void* y, int64_t ldy,
-                          bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
-                          void* stream) {
+static bro_status gemm_impl(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
+                            int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, bro_out_dtype out_dtype,
+                            void* workspace, size_t workspace_bytes, void* stream, bool w_static) {
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0 || ldy < N) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (out_dtype != BRO_OUT_BF16 && out_dtype != BRO_OUT_F32) return BRO_ERR_SHAPE;
@@ -322,7 +321,16 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
     return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, di.sm_count,
                               static_cast<cudaStream_t>(stream));
   return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,
-                           workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream));
+                           workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream), w_static);
+}
+
+bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* wcodes,
+                          const void* wscales, int64_t M, int64_t N, int64_t K, void* y, int64_t ldy,
+                          bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+  // the weights may have been written by the kernel just before this one: no early fetch
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, out_dtype, workspace, workspace_bytes, stream,
+                   false);
 }
 
 static bro_status linear_impl(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs,
@@ -340,8 +348,10 @@ static bro_status linear_impl(const void* x_bf16, int64_t M, int64_t K, int64_t 
   bro_status rc = launch_rotate_quantize(x_bf16, M, K, ldx, block, signs, acodes, ascales, BRO_LAYOUT_GEMM,
                                          static_cast<cudaStream_t>(stream));
   if (rc != BRO_OK) return rc;
-  return bro_gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
-                        bro_gemm_workspace_bytes(M, N, K), stream);
+  // The packed weights are older than the rotate+quantize kernel just enqueued, which signals its
+  // dependents only after its own wait: the GEMM may fetch its first weight tiles early.
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
+                   bro_gemm_workspace_bytes(M, N, K), stream, true);
 }
 
 bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,

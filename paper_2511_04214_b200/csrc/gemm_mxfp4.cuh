@@ -63,6 +63,7 @@ struct Params {
   int64_t kblocks;          // 512-byte scale blocks per 128-row block = 2*ceil(K/256)
   int num_k_steps;          // ceil(K/256)
   int tiles_m, tiles_n, total_tiles;
+  int w_static;             // the weight operand was complete before the previous kernel started (see launch)
 };
 
 // ---- tcgen05 wrappers ------------------------------------------------------------------------
@@ -451,7 +452,11 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   __syncthreads();
   tc_fence_after();
   griddep_launch_dependents();
-  griddep_wait();               // operands come from the kernel before; y may still be read by it
+  // Operands come from the kernel before, and y may still be read by it — except that in the
+  // whole-layer call the packed weights are older than that kernel, so the producer may start
+  // fetching the weight half of its first stages while the activations are still being written.
+  const bool early_w = p.w_static != 0 && warp == 0;
+  if (!early_w) griddep_wait();
   const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot_ptr, 0);
   const uint32_t tmem_sfa = tmem_base + C::kSfaCol;
   const uint32_t tmem_sfb = tmem_base + C::kSfbCol;
@@ -465,13 +470,42 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
       uint32_t phase = 0;
       int64_t issued = 0;
       bool ok = true;
+      int pre = 0;                  // K steps of the first tile whose loads are issued here
+      if (early_w) {
+        if ((int)blockIdx.x < p.total_tiles) {
+          const int tm = (int)blockIdx.x / p.tiles_n, tn = (int)blockIdx.x - tm * p.tiles_n;
+          const int m0 = tm * kBM, n0 = tn * BN;
+          const int nblk_valid = (BN == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1;
+          const uint8_t* sfa_src = p.ascales + (int64_t)tm * p.kblocks * 512;
+          const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
+          pre = p.num_k_steps < C::kStages ? p.num_k_steps : C::kStages;
+          for (int ks = 0; ks < pre; ++ks) {          // weights and their scales: before the wait
+            const uint32_t full = bar_full + 8 * ks;
+            mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
+            tma_load_2d(sB + ks * C::kBTileBytes, &tmw, ks * 128, n0, full);
+            for (int nb = 0; nb < nblk_valid; ++nb)
+              bulk_load_1d(sSFB + ks * C::kSfbBytes + nb * 1024, sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512,
+                           1024, full);
+          }
+          griddep_wait();
+          for (int ks = 0; ks < pre; ++ks) {          // activations and their scales: after it
+            const uint32_t full = bar_full + 8 * ks;
+            tma_load_2d(sA + ks * kATileBytes, &tma, ks * 128, m0, full);
+            bulk_load_1d(sSFA + ks * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
+          }
+          issued = pre;
+          if (pre == C::kStages) phase = 1u; else stage = pre;
+        } else {
+          griddep_wait();
+        }
+      }
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
         const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
         const int m0 = tm * kBM, n0 = tn * BN;
         const int nblk_valid = (BN == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1;
         const uint8_t* sfa_src = p.ascales + (int64_t)tm * p.kblocks * 512;
         const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
-        for (int ks = 0; ks < p.num_k_steps; ++ks) {
+        for (int ks = (tile == (int)blockIdx.x ? pre : 0); ks < p.num_k_steps; ++ks) {
           if (issued >= C::kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
           if (!ok) break;
           const uint32_t full = bar_full + 8 * stage;
@@ -556,9 +590,12 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
   return out_dtype == BRO_OUT_F32 ? go(gemm_mxfp4_kernel<BN, true>, 1) : go(gemm_mxfp4_kernel<BN, false>, 0);
 }
 
+// w_static: the caller guarantees that wcodes / wscales were complete before the kernel that
+// precedes this launch in the stream began (true inside the whole-layer calls, where that kernel is
+// the library's own rotate+quantize and signals its dependents only after its own wait).
 inline bro_status launch(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
                          int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* /*ws*/,
-                         size_t /*ws_bytes*/, int sm_count, cudaStream_t st) {
+                         size_t /*ws_bytes*/, int sm_count, cudaStream_t st, bool w_static = false) {
   int bn = 256;
   if (const char* e = getenv("BRO_GEMM_TILE_N")) bn = atoi(e) == 128 ? 128 : 256;
   else if (N <= 128) bn = 128;
@@ -569,6 +606,7 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   p.M = M; p.N = N; p.K = K; p.ldy = ldy;
   p.num_k_steps = (int)((K + kBK - 1) / kBK);
   p.kblocks = 2 * (int64_t)p.num_k_steps;
+  p.w_static = w_static ? 1 : 0;
   CUtensorMap tma, tmw, tmy;
   bro_status rc = make_codes_map(&tma, acodes, M, K, kBM);
   if (rc != BRO_OK) return rc;

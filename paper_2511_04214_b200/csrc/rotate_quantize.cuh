@@ -205,8 +205,9 @@ rotate_quantize_kernel(const __grid_constant__ CUtensorMap tmx, const Params p) 
     fence_proxy_async_smem();
   }
   __syncthreads();
-  griddep_launch_dependents();
   griddep_wait();               // x may be written, codes/scales still read, by the kernel before
+  // (only now: a dependent that starts early may then rely on everything older than this kernel)
+  griddep_launch_dependents();
 
   const int64_t total_tiles = p.tiles_m * p.tiles_k;
 

@@ -45,8 +45,9 @@ __global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(con
   const int ng = (int)(p.K >> 5);
   constexpr uint32_t cbits = rq::norm_bits<LOG2B>();
 
-  griddep_launch_dependents();
   griddep_wait();               // x may be written, codes/scales still read, by the kernel before
+  // (only now: a dependent that starts early may then rely on everything older than this kernel)
+  griddep_launch_dependents();
 
   // task -> (row, chunk); advanced incrementally (no division in the loop)
   int task = (int)blockIdx.x * kWarps + (int)(threadIdx.x >> 5);

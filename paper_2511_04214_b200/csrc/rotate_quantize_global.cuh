@@ -38,8 +38,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   const uint32_t cbits = (p.log2k % 2 == 0) ? (uint32_t)(127 - p.log2k / 2) << 23
                                             : 0x3FB504F3u - ((uint32_t)((p.log2k + 1) / 2) << 23);
   const int64_t row_iters = (p.M + p.rows_per_iter - 1) / p.rows_per_iter;
-  griddep_launch_dependents();
   griddep_wait();               // x may be written, codes/scales still read, by the kernel before
+  // (only now: a dependent that starts early may then rely on everything older than this kernel)
+  griddep_launch_dependents();
   // a thread always works on the same 32 channels, so its slice of the sign vector is loaded once
   uint4 sg[4] = {};
   if (p.signs) {
