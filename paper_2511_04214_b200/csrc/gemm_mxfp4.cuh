@@ -63,6 +63,10 @@ struct Params {
   int64_t kblocks;          // 512-byte scale blocks per 128-row block = 2*ceil(K/256)
   int num_k_steps;          // ceil(K/256)
   int tiles_m, tiles_n, total_tiles;
+  // Work units: units [0, full_units) are whole 128 x BN tiles in row-major tile order; when the
+  // tile count leaves the last round of the grid less than half full, the remaining tiles are cut
+  // into two 128 x BN/2 halves each (units full_units ..), so that the last round keeps every SM busy.
+  int full_units, total_units;
   int w_static;             // the weight operand was complete before the previous kernel started (see launch)
 };
 
@@ -219,6 +223,22 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// Unit index -> first row, first column and width of its output tile.
+template <int BN>
+__device__ __forceinline__ void decode_unit(const Params& p, int u, int& m0, int& n0, int& bn) {
+  int tile = u, half = 0;
+  bn = BN;
+  if (u >= p.full_units) {
+    const int idx = u - p.full_units;
+    tile = p.full_units + (idx >> 1);
+    half = idx & 1;
+    bn = BN / 2;
+  }
+  const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+  m0 = tm * kBM;
+  n0 = tn * BN + half * (BN / 2);
+}
+
 // Addresses the issuing warp works with (shared-memory window addresses of stage 0 and of the
 // first barrier of each kind).
 struct IssueRing {
@@ -236,14 +256,18 @@ struct IssueRing {
 template <int CG, int BN, int STAGES, int A_STAGE, int B_STAGE, int SFA_STAGE, int SFB_STAGE, int ACC_STRIDE,
           bool OVERLAP>
 __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem_base, uint32_t tmem_sfa,
-                                               uint32_t tmem_sfb, uint32_t idesc0, int my_tiles, int num_k_steps,
-                                               bool issue_lane) {
+                                               uint32_t tmem_sfb, uint32_t idesc_full, int my_tiles, int num_k_steps,
+                                               bool issue_lane, int narrow_from = 0x7FFFFFFF,
+                                               uint32_t idesc_narrow = 0u) {
+  // tiles narrow_from.. of this CTA are half-width: same loop, the instruction descriptor says N = BN/2
+  // (the scale copies still move both W row blocks; the second one is simply not read)
   const uint32_t issue = issue_lane ? 1u : 0u;
   const uint32_t a_lo0 = desc_lo_sw128(r.sA), b_lo0 = desc_lo_sw128(r.sB);
   const uint32_t sfa_lo0 = desc_lo_sf(r.sSFA), sfb_lo0 = desc_lo_sf(r.sSFB);
   const uint32_t hi_op = kDescHiSw128, hi_sf = kDescHiSf;
+  uint32_t idesc0 = idesc_full;
   // scale bytes {0,1} of a 32-bit scale word for the first MMA of a half, {2,3} for the second
-  const uint32_t idesc1 = idesc0 | (2u << 4) | (2u << 29);
+  uint32_t idesc1 = idesc0 | (2u << 4) | (2u << 29);
   auto copy_scales = [&](int stage, int h) {
     const uint32_t lo_a = sfa_lo0 + (uint32_t)stage * (SFA_STAGE >> 4) + (uint32_t)h * 32u;
     const uint32_t lo_b = sfb_lo0 + (uint32_t)stage * (SFB_STAGE >> 4) + (uint32_t)h * 32u;
@@ -278,6 +302,10 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
     if (!ok) break;
     tc_fence_after();
     const uint32_t tmem_acc = tmem_base + buf * ACC_STRIDE;
+    if (it >= narrow_from) {
+      idesc0 = idesc_narrow;
+      idesc1 = idesc0 | (2u << 4) | (2u << 29);
+    }
     for (int ks = 0; ks < num_k_steps; ++ks) {
       const bool has_next = (ks + 1 < num_k_steps) || (it + 1 < my_tiles);
       const int next_stage = (stage + 1 == STAGES) ? 0 : stage + 1;
@@ -408,7 +436,8 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
 template <int BN, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw,
-                  const __grid_constant__ CUtensorMap tmy, const Params p) {
+                  const __grid_constant__ CUtensorMap tmw_half, const __grid_constant__ CUtensorMap tmy,
+                  const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -466,61 +495,59 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
     if (lane == 0) {
       tma_prefetch_desc(&tma);
       tma_prefetch_desc(&tmw);
+      if (p.total_units > p.full_units) tma_prefetch_desc(&tmw_half);
       int stage = 0;
       uint32_t phase = 0;
       int64_t issued = 0;
       bool ok = true;
-      int pre = 0;                  // K steps of the first tile whose loads are issued here
-      if (early_w) {
-        if ((int)blockIdx.x < p.total_tiles) {
-          const int tm = (int)blockIdx.x / p.tiles_n, tn = (int)blockIdx.x - tm * p.tiles_n;
-          const int m0 = tm * kBM, n0 = tn * BN;
-          const int nblk_valid = (BN == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1;
-          const uint8_t* sfa_src = p.ascales + (int64_t)tm * p.kblocks * 512;
+      // loads of one K step of one unit; `part` selects the weight side (1), the activation side (2) or both (3)
+      auto issue_step = [&](int m0, int n0, int bn, int ks, int st, int part) {
+        // 128-row blocks of W scales that exist for this unit (a half-width unit of a ragged last
+        // tile can lie entirely beyond N: no block is read then, its columns are never stored)
+        const int nblk_valid = (int64_t)n0 >= p.N ? 0 : ((bn == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1);
+        const uint32_t full = bar_full + 8 * st;
+        if (part & 1) {
+          mbar_arrive_expect_tx(full, kATileBytes + bn * 128 + C::kSfaBytes + nblk_valid * 1024);
+          tma_load_2d(sB + st * C::kBTileBytes, bn == BN ? &tmw : &tmw_half, ks * 128, n0, full);
           const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
+          for (int nb = 0; nb < nblk_valid; ++nb)
+            bulk_load_1d(sSFB + st * C::kSfbBytes + nb * 1024, sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512, 1024,
+                         full);
+        }
+        if (part & 2) {
+          tma_load_2d(sA + st * kATileBytes, &tma, ks * 128, m0, full);
+          bulk_load_1d(sSFA + st * C::kSfaBytes, p.ascales + ((int64_t)(m0 / kBM) * p.kblocks + 2 * ks) * 512, 1024, full);
+        }
+      };
+      int pre = 0;                  // K steps of the first unit whose loads are issued here
+      if (early_w) {
+        if ((int)blockIdx.x < p.total_units) {
+          int m0, n0, bn;
+          decode_unit<BN>(p, (int)blockIdx.x, m0, n0, bn);
           pre = p.num_k_steps < C::kStages ? p.num_k_steps : C::kStages;
-          for (int ks = 0; ks < pre; ++ks) {          // weights and their scales: before the wait
-            const uint32_t full = bar_full + 8 * ks;
-            mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
-            tma_load_2d(sB + ks * C::kBTileBytes, &tmw, ks * 128, n0, full);
-            for (int nb = 0; nb < nblk_valid; ++nb)
-              bulk_load_1d(sSFB + ks * C::kSfbBytes + nb * 1024, sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512,
-                           1024, full);
-          }
+          for (int ks = 0; ks < pre; ++ks) issue_step(m0, n0, bn, ks, ks, 1);   // weights: before the wait
           griddep_wait();
-          for (int ks = 0; ks < pre; ++ks) {          // activations and their scales: after it
-            const uint32_t full = bar_full + 8 * ks;
-            tma_load_2d(sA + ks * kATileBytes, &tma, ks * 128, m0, full);
-            bulk_load_1d(sSFA + ks * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
-          }
+          for (int ks = 0; ks < pre; ++ks) issue_step(m0, n0, bn, ks, ks, 2);   // activations: after it
           issued = pre;
           if (pre == C::kStages) phase = 1u; else stage = pre;
         } else {
           griddep_wait();
         }
       }
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
-        const int m0 = tm * kBM, n0 = tn * BN;
-        const int nblk_valid = (BN == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1;
-        const uint8_t* sfa_src = p.ascales + (int64_t)tm * p.kblocks * 512;
-        const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
-        for (int ks = (tile == (int)blockIdx.x ? pre : 0); ks < p.num_k_steps; ++ks) {
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+        int m0, n0, bn;
+        decode_unit<BN>(p, u, m0, n0, bn);
+        for (int ks = (u == (int)blockIdx.x ? pre : 0); ks < p.num_k_steps; ++ks) {
           if (issued >= C::kStages) ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
           if (!ok) break;
-          const uint32_t full = bar_full + 8 * stage;
-          mbar_arrive_expect_tx(full, kATileBytes + C::kBTileBytes + C::kSfaBytes + nblk_valid * 1024);
-          tma_load_2d(sA + stage * kATileBytes, &tma, ks * 128, m0, full);
-          tma_load_2d(sB + stage * C::kBTileBytes, &tmw, ks * 128, n0, full);
-          bulk_load_1d(sSFA + stage * C::kSfaBytes, sfa_src + (int64_t)ks * 1024, 1024, full);
-          for (int nb = 0; nb < nblk_valid; ++nb)
-            bulk_load_1d(sSFB + stage * C::kSfbBytes + nb * 1024,
-                         sfb_src + ((int64_t)nb * p.kblocks + 2 * ks) * 512, 1024, full);
+          issue_step(m0, n0, bn, ks, stage, 3);
           ++issued;
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
+        // Do not leave while copies may still land in this CTA's shared memory: wait (bounded)
+        // for the last load armed on every stage.
         const int64_t first = issued > C::kStages ? issued - C::kStages : 0;
         for (int64_t i = first; i < issued; ++i)
           mbar_wait(bar_full + 8 * (int)(i % C::kStages), (uint32_t)((i / C::kStages) & 1), SITE_GEMM_DRAIN);
@@ -529,24 +556,32 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     const IssueRing ring = {sA, sB, sSFA, sSFB, bar_full, bar_empty, bar_acc_full, bar_acc_free, bar_ovl_free};
-    const int my_tiles =
-        (int)blockIdx.x < p.total_tiles ? (p.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    auto units_below = [&](int limit) {   // how many of this CTA's units have an index below `limit`
+      return (int)blockIdx.x < limit ? (limit - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    };
     mma_issue_loop<1, BN, C::kStages, kATileBytes, C::kBTileBytes, C::kSfaBytes, C::kSfbBytes, C::kAccStride,
-                   C::kOverlap>(ring, tmem_base, tmem_sfa, tmem_sfb, make_idesc<BN>(), my_tiles, p.num_k_steps,
-                                lane == 0);
+                   C::kOverlap>(ring, tmem_base, tmem_sfa, tmem_sfb, make_idesc<BN>(), units_below(p.total_units),
+                                p.num_k_steps, lane == 0, units_below(p.full_units), make_idesc<BN / 2>());
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
     int it = 0;
-    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++it) {
-      const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+    for (int u = blockIdx.x; u < p.total_units; u += gridDim.x, ++it) {
+      int m0, n0, bn;
+      decode_unit<BN>(p, u, m0, n0, bn);
       const int buf = it & 1;
       if (!mbar_wait_warp(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL)) break;
       tc_fence_after();
-      epilogue_tile<C::kChunks, C::kOverlap, OUT_F32>(
-          tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16), buf, lane, tm * kBM + q * 32, tn * BN, p.M, p.N,
-          p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u),
-          [&] { mbar_arrive(bar_ovl_free + 8 * buf); }, [&] { mbar_arrive(bar_acc_free + 8 * buf); });
+      const uint32_t tmem_acc = tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16);
+      const uint32_t stage_buf = sOut + (uint32_t)q * (32u * 128u);
+      auto release_shared = [&] { mbar_arrive(bar_ovl_free + 8 * buf); };
+      auto release_all = [&] { mbar_arrive(bar_acc_free + 8 * buf); };
+      if (bn == BN)
+        epilogue_tile<C::kChunks, C::kOverlap, OUT_F32>(tmem_acc, buf, lane, m0 + q * 32, n0, p.M, p.N, p.y, p.ldy, &tmy,
+                                                        stage_buf, release_shared, release_all);
+      else
+        epilogue_tile<C::kChunks / 2, C::kOverlap, OUT_F32>(tmem_acc, buf, lane, m0 + q * 32, n0, p.M, p.N, p.y, p.ldy,
+                                                            &tmy, stage_buf, release_shared, release_all);
     }
     // the staging buffer must have been read before this CTA's shared memory goes away; the writes
     // themselves complete with the kernel
@@ -563,16 +598,24 @@ bro_status make_codes_map(CUtensorMap* map, const void* base, int64_t rows, int6
 bro_status make_out_map(CUtensorMap* map, const void* y, int64_t M, int64_t N, int64_t ldy);
 
 template <int BN>
-bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUtensorMap& tmy, Params& p,
-                       int out_dtype, int sm_count, cudaStream_t st) {
+bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUtensorMap& tmw_half,
+                       const CUtensorMap& tmy, Params& p, int out_dtype, int sm_count, cudaStream_t st) {
   using C = Cfg<BN>;
   p.tiles_m = (int)((p.M + kBM - 1) / kBM);
   p.tiles_n = (int)((p.N + BN - 1) / BN);
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
-  if (total > 0x7FFFFFFF) return BRO_ERR_UNSUPPORTED;
+  if (total > 0x3FFFFFFF) return BRO_ERR_UNSUPPORTED;
   p.total_tiles = (int)total;
-  const int grid = (int)(total < sm_count ? total : sm_count);
-  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
+  // Rounds of the persistent grid: when the last round would leave at least half of the SMs idle,
+  // its tiles are cut into two half-width units each (BRO_GEMM_SPLIT=0 switches this off).
+  int64_t grid = total < sm_count ? total : sm_count;
+  const int64_t rem = total % sm_count;
+  bool split = BN == 256 && rem > 0 && 2 * rem <= sm_count;
+  if (const char* e = getenv("BRO_GEMM_SPLIT")) split = split && atoi(e) != 0;
+  p.full_units = (int)(split ? total - rem : total);
+  p.total_units = (int)(split ? total + rem : total);
+  if (split && p.total_units < sm_count) grid = p.total_units;
+  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
     static bool attr_done[64][2] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -582,7 +625,7 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
         return BRO_ERR_CUDA;
       attr_done[dev][which] = true;
     }
-    return cuda_ok(launch_kernel(kernel, (unsigned)grid, kThreads, C::kSmemBytes, st, 1, tma, tmw, tmy, p),
+    return cuda_ok(launch_kernel(kernel, (unsigned)grid, kThreads, C::kSmemBytes, st, 1, tma, tmw, tmw_half, tmy, p),
                    "gemm_mxfp4 launch")
                ? BRO_OK
                : BRO_ERR_CUDA;
@@ -618,8 +661,11 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   } else {
     tmy = tma;   // unused by the fp32-output kernel
   }
-  return bn == 256 ? launch_tile<256>(tma, tmw, tmy, p, out_dtype, sm_count, st)
-                   : launch_tile<128>(tma, tmw, tmy, p, out_dtype, sm_count, st);
+  CUtensorMap tmw_half;       // the same weights seen through a box of half as many rows
+  rc = make_codes_map(&tmw_half, wcodes, N, K, bn / 2);
+  if (rc != BRO_OK) return rc;
+  return bn == 256 ? launch_tile<256>(tma, tmw, tmw_half, tmy, p, out_dtype, sm_count, st)
+                   : launch_tile<128>(tma, tmw, tmw_half, tmy, p, out_dtype, sm_count, st);
 }
 
 }  // namespace gemm

@@ -139,6 +139,20 @@ def test_ragged_shapes(bro, tile_n, M, N, K):
     run_case(bro, ac, asc, wc, wsc)
 
 
+@pytest.mark.parametrize("M,N,K", [(128 * 19, 2048, 256), (128 * 5, 300, 512), (128 * 3, 4 * 256 + 40, 288)])
+def test_half_width_units_of_the_last_round(bro, M, N, K):
+    """Tile counts that leave the last round of the persistent grid less than half full (152 = 148 + 4
+    tiles; 10 and 15 tiles, fewer than half the SMs): the remaining tiles are computed as two
+    half-width units each.  Includes a ragged N whose last half-width unit lies beyond N."""
+    _, _, ac, asc, wc, wsc = quantized_pair(M, N, K, seed=M + N)
+    run_case(bro, ac, asc, wc, wsc)
+    os.environ["BRO_GEMM_SPLIT"] = "0"
+    try:
+        run_case(bro, ac, asc, wc, wsc)
+    finally:
+        del os.environ["BRO_GEMM_SPLIT"]
+
+
 def test_row_stride_of_y(bro, tile_n):
     _, _, ac, asc, wc, wsc = quantized_pair(130, 136, 256, seed=9)
     run_case(bro, ac, asc, wc, wsc, ldy=136 + 24)
