@@ -232,6 +232,9 @@ def run_ours(args):
     ring = max(2, min(8, -(-3 * L2_BYTES // per_step_bytes)))
     sets = []
     stream = torch.cuda.current_stream()
+    # --randomised: R_i = diag(s) H / sqrt(block) with a seeded +-1 vector per layer (Sec. 5.1)
+    signs = [synth.rotation_signs(K, seed=cfg["seed"] + idx[j]).to(dev) if args.randomised else None
+             for j, (M, K, N) in enumerate(shapes)]
     for j, (M, K, N) in enumerate(shapes):
         i = idx[j]
         w = synth.weights(N, K, seed=cfg["seed"] + i).to(dev)
@@ -241,7 +244,10 @@ def run_ours(args):
         for r in range(ring):
             wcodes = bro.alloc_codes(N, K, dev)
             wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM, dev)
-            bro.pack_weights(w, block, wcodes, wscales)                  # offline, untimed
+            if signs[j] is not None:
+                bro.pack_weights_rs(w, block, signs[j], wcodes, wscales)  # offline, untimed
+            else:
+                bro.pack_weights(w, block, wcodes, wscales)              # offline, untimed
             x = x0.to(dev).roll(r * 7, 0).contiguous()        # same statistics, separate memory
             per_ring.append({"x": x, "wcodes": wcodes, "wscales": wscales,
                              "y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
@@ -253,7 +259,10 @@ def run_ours(args):
     def step(r):
         for i, (M, K, N) in enumerate(shapes):
             s = sets[i][r % ring]
-            bro.linear(s["x"], block, s["wcodes"], s["wscales"], N, s["y"], s["ws"])
+            if signs[i] is not None:
+                bro.linear_rs(s["x"], block, signs[i], s["wcodes"], s["wscales"], N, s["y"], s["ws"])
+            else:
+                bro.linear(s["x"], block, s["wcodes"], s["wscales"], N, s["y"], s["ws"])
 
     flops_per_step = sum(2.0 * M * K * N for (M, K, N) in shapes)
     sampler = ClockSampler(local_rank)
@@ -326,7 +335,10 @@ def run_ours(args):
             ev[0].record()
             for r in range(ring):
                 s, acodes, ascales = views(i, r)
-                bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
+                if signs[i] is not None:
+                    bro.rotate_quantize_mxfp4_rs(s["x"], block, signs[i], acodes, ascales, bro.LAYOUT_GEMM)
+                else:
+                    bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
             ev[1].record()
             for r in range(ring):
                 s, acodes, ascales = views(i, r)
@@ -347,7 +359,7 @@ def run_ours(args):
 
     # ---- end-to-end through the host-buffer entry point
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.randomised:     # (the host-buffer entry point has no randomised form)
         host = []
         for i, (M, K, N) in enumerate(shapes):
             s = sets[i][0]
@@ -397,7 +409,8 @@ def run_ours(args):
             "dtype": "mxfp4 (e2m1 x e8m0) operands, f32 accumulate, bf16 out", "data": "synthetic",
             "config": {"workload": args.workload, "shapes_MKN": shapes, "block": block,
                        "l2": f"ring of {ring} independent input/output sets ({per_step_bytes * ring / 1e6:.0f} MB) > 126 MB L2",
-                       "launch": "cuda_graph" if graph is not None else "direct", "parallelism": "replicas only"},
+                       "launch": "cuda_graph" if graph is not None else "direct", "parallelism": "replicas only",
+                       "rotation": "randomised block Hadamard (diag(s) H)" if args.randomised else "block Hadamard"},
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": steps * len(shapes) * 2,
@@ -472,6 +485,26 @@ def run_rotate_quantize_only(args):
         ts = [a.elapsed_time(c) / group for a, c in evs[b]]
         per_block[str(b if b else K)] = {"us": statistics.mean(ts) * 1e3, "gbs": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9,
                                          "frac_of_measured_copy": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    # The oracle's per-group quantisation error per rotation size (Sec. 4.1 / 4.2, Fig. 6-7), on the
+    # first 512 rows: mean over all MX groups, and split into regular and outlier groups (a group
+    # is an outlier group if it holds one of the top 0.1 % |x| entries of the sample).
+    oracle_mse = None
+    if not args.no_cpu_baseline:
+        import numpy as np
+        import oracle
+        rows = 512
+        xs_cpu = synth.activations(M, K, seed=cfg["seed"], recipe=cfg["recipe"])[:rows]
+        bits = synth.bf16_bits(xs_cpu)
+        absx = np.abs(xs_cpu.float().numpy())
+        thresh = np.quantile(absx, 0.999)
+        outlier = (absx.reshape(rows, K // 32, 32) >= thresh).any(-1)
+        oracle_mse = {"rows": rows, "outlier_group_fraction": float(outlier.mean())}
+        for b in blocks:
+            y = oracle.rotate(bits, b)
+            c, sc = oracle.quantize(y)
+            mse = oracle.group_mse(y, c, sc)
+            oracle_mse[str(b if b else K)] = {"all": float(mse.mean()), "regular": float(mse[~outlier].mean()),
+                                              "outlier": float(mse[outlier].mean())}
     ms_total = t_all0.elapsed_time(t_all1)
     value = bytes_per_launch * len(blocks) * steps / (ms_total * 1e-3) / 1e9
     first = per_block[str(blocks[0] if blocks[0] else K)]
@@ -481,6 +514,7 @@ def run_rotate_quantize_only(args):
            "config": {"workload": "cfg4", "shape_MK": [M, K], "blocks": [b if b else K for b in blocks],
                       "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm"},
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
+           "oracle_group_mse": oracle_mse,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                         "traffic": None, "algorithmic_bytes": bytes_per_launch,
@@ -501,6 +535,8 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=0,
                     help="rows per shape per step for --impl reference (0 = sized to finish in ~2 min)")
     ap.add_argument("--only-block", action="store_true", help="cfg4: run only --block instead of the sweep")
+    ap.add_argument("--randomised", action="store_true",
+                    help="use the randomised block rotation diag(s) H / sqrt(block) (the *_rs entry points)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
