@@ -505,6 +505,30 @@ def run_rotate_quantize_only(args):
             mse = oracle.group_mse(y, c, sc)
             oracle_mse[str(b if b else K)] = {"all": float(mse.mean()), "regular": float(mse[~outlier].mean()),
                                               "outlier": float(mse[outlier].mean())}
+    # The same statistic over the WHOLE tensor on the GPU (bro_group_quant_error), timed the same way:
+    # 2 bytes read per element, 4 bytes written per group.
+    gpu_mse = {}
+    mse_buf = torch.empty((M, K // 32), dtype=torch.float32, device="cuda")
+    absx0 = xs[0].abs()
+    # outlier groups: hold one of the top 0.1 % |x| entries (threshold from the first 16 M entries)
+    sample = absx0.float().flatten()[: 1 << 24]
+    thresh_gpu = torch.kthvalue(sample, int(sample.numel() * 0.999)).values
+    outlier_gpu = (absx0.view(M, K // 32, 32) >= thresh_gpu).any(-1)
+    for b in blocks:
+        for i in range(3):
+            bro.group_quant_error(xs[i % ring], b, mse_buf)
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(2 * ring):
+            bro.group_quant_error(xs[i % ring], b, mse_buf)
+        c.record()
+        bro.group_quant_error(xs[0], b, mse_buf)
+        torch.cuda.synchronize()
+        us = a.elapsed_time(c) * 1e3 / (2 * ring)
+        gpu_mse[str(b if b else K)] = {"us": us, "gbs": M * K * 2.125 / us / 1e3, "all": float(mse_buf.mean()),
+                                       "regular": float(mse_buf[~outlier_gpu].mean()),
+                                       "outlier": float(mse_buf[outlier_gpu].mean())}
+    assert bro.last_device_status() == 0
     ms_total = t_all0.elapsed_time(t_all1)
     value = bytes_per_launch * len(blocks) * steps / (ms_total * 1e-3) / 1e9
     first = per_block[str(blocks[0] if blocks[0] else K)]
@@ -514,7 +538,7 @@ def run_rotate_quantize_only(args):
            "config": {"workload": "cfg4", "shape_MK": [M, K], "blocks": [b if b else K for b in blocks],
                       "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm"},
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
-           "oracle_group_mse": oracle_mse,
+           "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                         "traffic": None, "algorithmic_bytes": bytes_per_launch,

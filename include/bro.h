@@ -158,6 +158,20 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
                          void* stream);
 
 /*
+ * Analysis: the quantisation error the rotation leaves per MX group (Sec. 4.1-4.2 and Fig. 3 / 6:
+ * error of regular vs. outlier blocks under the shared power-of-two scale; App. A.3).  For every
+ * row of x and every group of 32 channels of y = x R_block:
+ *   mse[m, g] = mean_i (y_i - deq(Q(y))_i)^2
+ * with Q the MXFP4 quantiser of bro_rotate_quantize_mxfp4.  Nothing else is written.
+ *   block       32, 64, 128 or 0 (= K), as above;  signs_bf16  NULL or the +-1 vector of the
+ *               randomised rotation;  mse  device, fp32 [M, K/32], dense.
+ * Arithmetic: differences are exact, squares and their sum are rounded in fp32 (relative error of a
+ * few 2^-24 against an fp64 evaluation).
+ */
+bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                 const void* signs_bf16, float* mse, void* stream);
+
+/*
  * bro_linear for a caller whose activations and result live in HOST memory (pinned memory gives
  * asynchronous copies).  Copies x_host[M, K] (dense, ldx = K) to the device staging buffer,
  * runs bro_linear, and copies y[M, N] (dense) back to y_host, all on `stream`.

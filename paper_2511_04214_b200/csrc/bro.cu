@@ -146,7 +146,7 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   if (rc != BRO_OK) return rc;
 
   if (B > 128) {
-    return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, layout, gemm_scale_kblocks(K), di.sm_count, st);
+    return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, nullptr, layout, gemm_scale_kblocks(K), di.sm_count, st);
   }
 
   // Register-streaming kernel by default; BRO_RQ_TMA=1 selects the TMA-ring kernel (also used when
@@ -281,6 +281,27 @@ bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K
                                         void* stream) {
   return launch_rotate_quantize(x_bf16, M, K, ldx, block, signs_bf16, codes, scales, layout,
                                 static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                 const void* signs_bf16, float* mse, void* stream) {
+  if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (M == 0) return BRO_OK;
+  if (!x_bf16 || !mse) return BRO_ERR_NULL;
+  const int64_t B = block == 0 ? K : block;
+  if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  if (K % B != 0) return BRO_ERR_SHAPE;
+  if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
+  if (ldx % 8 != 0 || !aligned(x_bf16, 16) || !aligned(mse, 4) || !aligned(signs_bf16, 16)) return BRO_ERR_ALIGN;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (B > 128)
+    return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
+  if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
+  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, mse, di.sm_count, st);
 }
 
 bro_status bro_pack_weights_rs(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,

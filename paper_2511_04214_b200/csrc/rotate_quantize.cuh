@@ -20,6 +20,8 @@
 //    the tile are gathered with two shuffles and written as one 32-bit store.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "bro_common.cuh"
 
 namespace bro {
@@ -182,6 +184,39 @@ __device__ __forceinline__ uint32_t quantize_group(const uint64_t (&P)[16], uint
     w[j] = pack_e2m1x8(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3], r[8 * j + 4], r[8 * j + 5],
                        r[8 * j + 6], r[8 * j + 7]);
   return s;
+}
+
+// Quantisation error of one MX group (paper Sec. 4.1-4.2: block-level error under the shared
+// power-of-two scale): mean over the 32 elements of (y - deq(Q(y)))^2 with y = v * c the rotated
+// values.  The codes are produced by the same conversion instruction as in quantize_group and
+// decoded again in hardware (e2m1x2 -> f16x2); in the scaled domain r = y * 2^-E the difference
+// r - q is exact in fp32, squares and their sum are rounded in fp32, the result is rescaled by 2^2E.
+__device__ __forceinline__ float group_error(const uint64_t (&P)[16], uint32_t cbits) {
+  const float c = __uint_as_float(cbits);
+  const uint64_t cc = pack2(c, c);
+  float y[32];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) unpack2(mul2(P[k], cc), y[2 * k], y[2 * k + 1]);
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(y[i]));
+  const uint32_t ef = __float_as_uint(m) >> 23;
+  const uint32_t s = ef > 2u ? ef - 2u : 0u;
+  const float inv = __uint_as_float((254u - s) << 23);                    // 2^-E, E = s - 127
+  const float pe = __uint_as_float(s >= 1u ? (s << 23) : 0x00400000u);    // 2^E (2^-127 is subnormal)
+  float acc = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    const float r0 = __fmul_rn(y[i], inv), r1 = __fmul_rn(y[i + 1], inv);
+    uint32_t h;
+    asm("{ .reg .b8 b; cvt.rn.satfinite.e2m1x2.f32 b, %2, %1; cvt.rn.f16x2.e2m1x2 %0, b; }" : "=r"(h) : "f"(r0), "f"(r1));
+    const float q0 = __half2float(__ushort_as_half((unsigned short)(h & 0xFFFFu)));
+    const float q1 = __half2float(__ushort_as_half((unsigned short)(h >> 16)));
+    const float d0 = __fsub_rn(r0, q0), d1 = __fsub_rn(r1, q1);
+    acc = __fadd_rn(acc, __fmul_rn(d0, d0));
+    acc = __fadd_rn(acc, __fmul_rn(d1, d1));
+  }
+  return __fmul_rn(__fmul_rn(__fmul_rn(acc, 0.03125f), pe), pe);
 }
 
 // SIGNS: the randomised rotation R_i = diag(s) H / sqrt(block) (paper Sec. 5.1) — the channel signs

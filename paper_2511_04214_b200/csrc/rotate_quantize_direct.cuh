@@ -36,9 +36,12 @@ struct Params {
   int groups_padded;            // groups per row it covers (scale padding included)
   int chunks_per_row;           // ceil(groups_padded / 32)
   int total_tasks;              // rows_padded * chunks_per_row; one task = one warp, 32 groups of a row
+  float* mse;                   // STATS kernels: [M, K/32] per-group quantisation error instead of codes/scales
 };
 
-template <int LOG2B, bool SIGNS>
+// STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
+// (rq::group_error) — the analysis behind the paper's regular-block / outlier-block comparison.
+template <int LOG2B, bool SIGNS, bool STATS>
 __global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(const Params p) {
   const int lane = threadIdx.x & 31;
   const int num_warps = (int)gridDim.x * kWarps;
@@ -86,11 +89,20 @@ __global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(con
     rq::fwht32_stages_2_to_16(P);
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
-    uint32_t w[4];
-    const uint32_t s = rq::quantize_group(P, cbits, w);
-
     const int g = chunk * 32 + lane;
     const bool live = row < p.M && g < ng;
+    if (STATS) {
+      const float e = rq::group_error(P, cbits);
+      if (live) p.mse[(int64_t)row * ng + g] = e;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+      task = ntask;
+      row = nrow;
+      chunk = nchunk;
+      continue;
+    }
+    uint32_t w[4];
+    const uint32_t s = rq::quantize_group(P, cbits, w);
     if (live)
       *reinterpret_cast<uint4*>(p.codes + (int64_t)row * (p.K >> 1) + (int64_t)g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
     // scale bytes of 4 consecutive groups -> one 32-bit word in the lane with g % 4 == 0
@@ -126,9 +138,9 @@ inline bool supports(int64_t M, int64_t K, bro_layout layout, int64_t scale_kblo
   return rows * ((groups + 31) / 32) < ((int64_t)1 << 30);
 }
 
-template <int LOG2B, bool SIGNS>
+template <int LOG2B, bool SIGNS, bool STATS>
 inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
-  auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS>;
+  auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS, STATS>;
   static int blocks_per_sm[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -145,6 +157,22 @@ inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
                                                                                                        : BRO_ERR_CUDA;
 }
 
+template <bool STATS>
+inline bro_status launch_any(Params& p, int log2b, int sm_count, cudaStream_t st) {
+  if (p.signs) {
+    switch (log2b) {
+      case 5: return launch_one<5, true, STATS>(p, sm_count, st);
+      case 6: return launch_one<6, true, STATS>(p, sm_count, st);
+      default: return launch_one<7, true, STATS>(p, sm_count, st);
+    }
+  }
+  switch (log2b) {
+    case 5: return launch_one<5, false, STATS>(p, sm_count, st);
+    case 6: return launch_one<6, false, STATS>(p, sm_count, st);
+    default: return launch_one<7, false, STATS>(p, sm_count, st);
+  }
+}
+
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs, void* codes,
                          void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
   Params p;
@@ -155,22 +183,31 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int l
   p.scale_kblocks = scale_kblocks;
   p.layout = (int)layout;
   p.signs = static_cast<const uint16_t*>(signs);
+  p.mse = nullptr;
   p.rows_padded = (int)(layout == BRO_LAYOUT_GEMM ? (M + 127) / 128 * 128 : M);
   p.groups_padded = (int)(layout == BRO_LAYOUT_GEMM ? scale_kblocks * 4 : K / 32);
   p.chunks_per_row = (p.groups_padded + 31) / 32;
   p.total_tasks = p.rows_padded * p.chunks_per_row;
-  if (signs) {
-    switch (log2b) {
-      case 5: return launch_one<5, true>(p, sm_count, st);
-      case 6: return launch_one<6, true>(p, sm_count, st);
-      default: return launch_one<7, true>(p, sm_count, st);
-    }
-  }
-  switch (log2b) {
-    case 5: return launch_one<5, false>(p, sm_count, st);
-    case 6: return launch_one<6, false>(p, sm_count, st);
-    default: return launch_one<7, false>(p, sm_count, st);
-  }
+  return launch_any<false>(p, log2b, sm_count, st);
+}
+
+// Per-group quantisation error only: mse[M, K/32] (fp32).
+inline bro_status launch_stats(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs,
+                               float* mse, int sm_count, cudaStream_t st) {
+  Params p;
+  p.x = static_cast<const uint16_t*>(x);
+  p.M = M; p.K = K; p.ldx = ldx;
+  p.codes = nullptr;
+  p.scales = nullptr;
+  p.scale_kblocks = 0;
+  p.layout = (int)BRO_LAYOUT_CANONICAL;
+  p.signs = static_cast<const uint16_t*>(signs);
+  p.mse = mse;
+  p.rows_padded = (int)M;
+  p.groups_padded = (int)(K / 32);
+  p.chunks_per_row = (p.groups_padded + 31) / 32;
+  p.total_tasks = p.rows_padded * p.chunks_per_row;
+  return launch_any<true>(p, log2b, sm_count, st);
 }
 
 }  // namespace rqd

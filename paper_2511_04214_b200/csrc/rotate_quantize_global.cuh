@@ -27,6 +27,7 @@ struct Params {
   int threads_per_row;   // K / 32
   int rows_per_iter;     // blockDim.x / threads_per_row
   const uint16_t* signs; // [K] bf16 +-1 for the randomised rotation diag(s) H / sqrt(K), or nullptr
+  float* mse;            // if set: write the per-group quantisation error [M, K/32] instead of codes/scales
 };
 
 template <int kMaxThreads>
@@ -92,6 +93,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
         P[2 * c + 1] = rq::pack2(__fmaf_rn(a2, sgn, o.z), __fmaf_rn(a3, sgn, o.w));
       }
     }
+    if (p.mse) {                 // analysis mode (uniform over the grid)
+      const float e = rq::group_error(P, cbits);
+      if (live) p.mse[row * (p.K >> 5) + gi] = e;
+      continue;
+    }
     uint32_t w[4];
     const uint32_t s = rq::quantize_group(P, cbits, w);
     if (live) {
@@ -109,7 +115,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
 }
 
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
-                         void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+                         void* scales, float* mse, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M;
@@ -120,6 +126,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   p.scale_kblocks = scale_kblocks;
   p.layout = (int)layout;
   p.signs = static_cast<const uint16_t*>(signs);
+  p.mse = mse;
   int lg = 0;
   while (((int64_t)1 << lg) < K) ++lg;
   p.log2k = lg;
@@ -127,7 +134,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   int threads = p.threads_per_row < 256 ? 256 : p.threads_per_row;
   p.rows_per_iter = threads / p.threads_per_row;
   const size_t smem = K > 1024 ? (size_t)p.rows_per_iter * K * sizeof(float) : 0;
-  if (layout == BRO_LAYOUT_GEMM) {
+  if (layout == BRO_LAYOUT_GEMM && !mse) {
     // padding rows / groups of the tiled scale buffer must read as 0
     const size_t bytes = (size_t)((M + 127) / 128) * (size_t)scale_kblocks * 512;
     if (cudaMemsetAsync(scales, 0, bytes, st) != cudaSuccess) return BRO_ERR_CUDA;
