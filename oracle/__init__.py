@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.bro_ref_gemm_mxfp4_points.argtypes = [p, p, p, p, i64, i64, i64, p, p, i64, p, p]
         L.bro_ref_linear.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, p]
         L.bro_ref_group_mse.argtypes = [p, p, p, i64, i64, p]
+        L.bro_ref_fake_quantize.argtypes = [p, i64, i64, ci, p]
+        L.bro_ref_fake_quantize.restype = ci
         for name in ("rotate_rs", "rotate_quantize_mxfp4_rs", "rotate", "quantize", "decode", "rotate_quantize_mxfp4", "pack_weights",
                      "gemm_mxfp4", "gemm_mxfp4_points", "linear", "group_mse"):
             getattr(L, "bro_ref_" + name).restype = ci
@@ -211,3 +213,23 @@ def group_mse(y, codes, scales) -> np.ndarray:
     _check(lib().bro_ref_group_mse(_ptr(y), _ptr(codes), _ptr(scales), rows, K, _ptr(mse)),
            "group_mse")
     return mse
+
+
+FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3}
+
+
+def fake_quantize(y, fmt) -> np.ndarray:
+    """Dequantised values (fp64) of fp32 rows under one of the compared 4-bit formats."""
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    rows, K = y.shape
+    out = np.empty((rows, K), dtype=np.float64)
+    f = FORMATS[fmt] if isinstance(fmt, str) else int(fmt)
+    _check(lib().bro_ref_fake_quantize(_ptr(y), rows, K, f, _ptr(out)), "fake_quantize")
+    return out
+
+
+def group_error(y, fmt) -> np.ndarray:
+    """mean_i (y_i - deq_i)^2 per group of 32, fp64, for any of the compared formats."""
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    d = y.astype(np.float64) - fake_quantize(y, fmt)
+    return (d * d).reshape(y.shape[0], y.shape[1] // MX_GROUP, MX_GROUP).mean(-1)

@@ -306,3 +306,71 @@ int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scale
     }
   return 0;
 }
+
+/* ---- comparison formats (analysis only) -------------------------------------------------------- */
+
+/* fp32 -> nearest-even fp16 value, returned as a float; clamped to the largest finite fp16. */
+static float round_to_fp16(float f) {
+  if (!(f == f)) return f;
+  float a = fabsf(f);
+  if (a >= 65520.0f) a = 65504.0f; /* would round to infinity: saturate */
+  else if (a < 6.103515625e-05f) { /* below 2^-14: fp16 subnormals, spacing 2^-24 */
+    a = (float)(rint((double)a * 16777216.0) / 16777216.0);
+  } else {
+    int e;
+    (void)frexpf(a, &e); /* a = m * 2^e, m in [0.5, 1): 11 significant bits -> spacing 2^(e-11) */
+    double q = ldexp(1.0, e - 11);
+    a = (float)(rint((double)a / q) * q);
+  }
+  return f < 0 ? -a : a;
+}
+
+int bro_ref_fake_quantize(const float* y, int64_t rows, int64_t K, int format, double* deq) {
+  if (!y || !deq) return 1;
+  if (rows < 0 || K <= 0 || K % MX_GROUP != 0 || format < 0 || format > 3) return 2;
+  const int64_t ng = K / MX_GROUP;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t g = 0; g < ng; ++g) {
+      const float* v = y + r * K + g * MX_GROUP;
+      double* out = deq + r * K + g * MX_GROUP;
+      float amax = 0.0f;
+      for (int i = 0; i < MX_GROUP; ++i)
+        if (fabsf(v[i]) > amax) amax = fabsf(v[i]);
+      const int ef = (int)((f32_bits(amax) >> 23) & 0xFF);
+      if (format == 0 || format == 2) {
+        /* power-of-two scale: MXFP4 keeps 2 integer bits above the scale, MXINT4 none */
+        int s = format == 0 ? ef - 2 : ef;
+        if (s < 0) s = 0;
+        const int E = s - 127;
+        for (int i = 0; i < MX_GROUP; ++i) {
+          const float rr = ldexpf(fabsf(v[i]), -E);
+          double q;
+          if (format == 0) q = E2M1_GRID[e2m1_round(rr)];
+          else {
+            double k = rint((double)rr * 4.0); /* exact product, ties to even */
+            if (k > 7.0) k = 7.0;
+            q = k / 4.0;
+          }
+          q = ldexp(q, E);
+          out[i] = (f32_bits(v[i]) >> 31) ? -q : q;
+        }
+      } else {
+        const float qmax = format == 1 ? 6.0f : 7.0f;
+        const float sc = round_to_fp16(amax / qmax); /* fp32 division, then fp16 rounding */
+        for (int i = 0; i < MX_GROUP; ++i) {
+          if (sc == 0.0f) { out[i] = 0.0; continue; }
+          const float rr = fabsf(v[i]) / sc; /* fp32 division */
+          double q;
+          if (format == 1) q = E2M1_GRID[e2m1_round(rr)];
+          else {
+            q = rint((double)rr);
+            if (q > 7.0) q = 7.0;
+          }
+          q *= (double)sc;
+          out[i] = (f32_bits(v[i]) >> 31) ? -q : q;
+        }
+      }
+    }
+  return 0;
+}

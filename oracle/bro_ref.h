@@ -105,6 +105,18 @@ int bro_ref_linear(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, in
 int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scales,
                       int64_t rows, int64_t K, double* mse);
 
+/* The 4-bit formats the paper compares MXFP4 with (Sec. 3.1, Sec. 3.2 / Fig. 2, Sec. 4.1 / Fig. 3),
+ * all symmetric, group of 32, applied to fp32 rows y:
+ *   0 MXFP4   E2M1 elements, E8M0 scale 2^E, E = floor(log2 amax) - 2           (as bro_ref_quantize)
+ *   1 BFP4    E2M1 elements, FP16 scale s = fp16(amax / 6)                       ("FP4 variant of BINT4")
+ *   2 MXINT4  INT4 elements k/4, k in [-7, 7], E8M0 scale 2^E, E = floor(log2 amax)
+ *   3 BINT4   INT4 elements k in [-7, 7], FP16 scale s = fp16(amax / 7)          (RTN, block 32, FP16 scale)
+ * The paper names the formats but gives no formulas; the scale and rounding rules above are this
+ * build's reading (round to nearest even everywhere, saturating; fp16 scale = the fp32 quotient
+ * rounded to nearest-even fp16, clamped to the largest finite fp16; a zero scale gives all zeros).
+ * Writes the dequantised values (exact in fp64) to deq[rows, K]. */
+int bro_ref_fake_quantize(const float* y, int64_t rows, int64_t K, int format, double* deq);
+
 #ifdef __cplusplus
 }
 #endif
