@@ -528,6 +528,15 @@ def run_rotate_quantize_only(args):
         gpu_mse[str(b if b else K)] = {"us": us, "gbs": M * K * 2.125 / us / 1e3, "all": float(mse_buf.mean()),
                                        "regular": float(mse_buf[~outlier_gpu].mean()),
                                        "outlier": float(mse_buf[outlier_gpu].mean())}
+    # Format study (Sec. 3.2 / Fig. 2-3) on the same tensor: mean group error per 4-bit format for the
+    # block-32 and the full-dimension rotation.
+    format_study = {}
+    for fmt in ("mxfp4", "bfp4", "mxint4", "bint4"):
+        format_study[fmt] = {}
+        for b in (32, 0):
+            bro.group_quant_error(xs[0], b, mse_buf, fmt=fmt)
+            format_study[fmt][str(b if b else K)] = {"all": float(mse_buf.mean()), "regular": float(mse_buf[~outlier_gpu].mean()),
+                                                     "outlier": float(mse_buf[outlier_gpu].mean())}
     assert bro.last_device_status() == 0
     ms_total = t_all0.elapsed_time(t_all1)
     value = bytes_per_launch * len(blocks) * steps / (ms_total * 1e-3) / 1e9
@@ -538,7 +547,7 @@ def run_rotate_quantize_only(args):
            "config": {"workload": "cfg4", "shape_MK": [M, K], "blocks": [b if b else K for b in blocks],
                       "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm"},
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
-           "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse,
+           "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse, "gpu_format_study": format_study,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                         "traffic": None, "algorithmic_bytes": bytes_per_launch,

@@ -64,6 +64,8 @@ typedef enum {
 
 typedef enum { BRO_LAYOUT_CANONICAL = 0, BRO_LAYOUT_GEMM = 1 } bro_layout;
 typedef enum { BRO_OUT_BF16 = 0, BRO_OUT_F32 = 1 } bro_out_dtype;
+/* 4-bit formats of the analysis entry point (see bro_group_quant_error_fmt). */
+typedef enum { BRO_FMT_MXFP4 = 0, BRO_FMT_BFP4 = 1, BRO_FMT_MXINT4 = 2, BRO_FMT_BINT4 = 3 } bro_format;
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* bro_status_string(bro_status s);
@@ -170,6 +172,21 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
  */
 bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                  const void* signs_bf16, float* mse, void* stream);
+
+/*
+ * The same statistic for the 4-bit formats the paper compares MXFP4 with (Sec. 3.1 BINT4 baseline;
+ * Sec. 3.2 / Fig. 2 format study; Sec. 4.1 / Fig. 3 MXFP4 against BFP4), all symmetric with groups
+ * of 32 and round to nearest even, saturating:
+ *   BRO_FMT_MXFP4   E2M1 elements, scale 2^E, E = floor(log2 amax) - 2
+ *   BRO_FMT_BFP4    E2M1 elements, FP16 scale fp16(amax / 6)
+ *   BRO_FMT_MXINT4  elements k/4 with |k| <= 7, scale 2^E, E = floor(log2 amax)
+ *   BRO_FMT_BINT4   integer elements |k| <= 7, FP16 scale fp16(amax / 7)
+ * (the paper names these formats without formulas; the rules above are this library's reading).
+ * Only MXFP4 has a GEMM here — the other formats exist for the error analysis.
+ */
+bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                     const void* signs_bf16, bro_format format, float* mse,
+                                     void* stream);
 
 /*
  * bro_linear for a caller whose activations and result live in HOST memory (pinned memory gives

@@ -25,7 +25,7 @@ EXPORTS = [
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host", "bro_linear_static",
-    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error",
+    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt",
 ]
 
 
@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     L.bro_linear_rs.argtypes = [p, i64, i64, i64, ci, p, p, p, i64, p, i64, p, sz, p]
     L.bro_group_quant_error.restype = ci
     L.bro_group_quant_error.argtypes = [p, i64, i64, i64, ci, p, p, p]
+    L.bro_group_quant_error_fmt.restype = ci
+    L.bro_group_quant_error_fmt.argtypes = [p, i64, i64, i64, ci, p, ci, p, p]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
     return L
@@ -243,11 +245,14 @@ def linear_rs(x: torch.Tensor, block: int, signs: torch.Tensor, wcodes, wscales,
            "bro_linear_rs")
 
 
+FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3}
+
+
 def group_quant_error(x: torch.Tensor, block: int, mse: torch.Tensor, signs: torch.Tensor = None,
-                      stream=None) -> None:
+                      stream=None, fmt: str = "mxfp4") -> None:
     """Per-group quantisation error of the rotated activations: ``mse`` is fp32 [M, K/32]."""
     assert x.dtype == torch.bfloat16 and mse.dtype == torch.float32 and mse.is_contiguous()
     M, K = x.shape
     assert mse.shape == (M, K // 32)
-    _check(lib.bro_group_quant_error(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), _ptr(mse), _stream(stream)),
-           "bro_group_quant_error")
+    _check(lib.bro_group_quant_error_fmt(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(mse),
+                                         _stream(stream)), "bro_group_quant_error_fmt")

@@ -146,7 +146,7 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   if (rc != BRO_OK) return rc;
 
   if (B > 128) {
-    return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, nullptr, layout, gemm_scale_kblocks(K), di.sm_count, st);
+    return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, nullptr, 0, layout, gemm_scale_kblocks(K), di.sm_count, st);
   }
 
   // Register-streaming kernel by default; BRO_RQ_TMA=1 selects the TMA-ring kernel (also used when
@@ -283,8 +283,9 @@ bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K
                                 static_cast<cudaStream_t>(stream));
 }
 
-bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
-                                 const void* signs_bf16, float* mse, void* stream) {
+bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                     const void* signs_bf16, bro_format format, float* mse, void* stream) {
+  if ((int)format < 0 || (int)format > 3) return BRO_ERR_SHAPE;
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (M == 0) return BRO_OK;
@@ -299,9 +300,14 @@ bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64
   if (rc != BRO_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (B > 128)
-    return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
+    return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, (int)format, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
   if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
-  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, mse, di.sm_count, st);
+  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, (int)format, mse, di.sm_count, st);
+}
+
+bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                 const void* signs_bf16, float* mse, void* stream) {
+  return bro_group_quant_error_fmt(x_bf16, M, K, ldx, block, signs_bf16, BRO_FMT_MXFP4, mse, stream);
 }
 
 bro_status bro_pack_weights_rs(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,

@@ -186,37 +186,80 @@ __device__ __forceinline__ uint32_t quantize_group(const uint64_t (&P)[16], uint
   return s;
 }
 
-// Quantisation error of one MX group (paper Sec. 4.1-4.2: block-level error under the shared
-// power-of-two scale): mean over the 32 elements of (y - deq(Q(y)))^2 with y = v * c the rotated
-// values.  The codes are produced by the same conversion instruction as in quantize_group and
-// decoded again in hardware (e2m1x2 -> f16x2); in the scaled domain r = y * 2^-E the difference
-// r - q is exact in fp32, squares and their sum are rounded in fp32, the result is rescaled by 2^2E.
-__device__ __forceinline__ float group_error(const uint64_t (&P)[16], uint32_t cbits) {
+// Quantisation error of one group of 32 (paper Sec. 4.1-4.2: block-level error under the shared
+// scale; Sec. 3.2 / Fig. 2-3 for the formats compared): mean over the group of (y - deq(Q(y)))^2 with
+// y = v * c the rotated values.  `format`: 0 MXFP4 (E2M1, scale 2^E, E = floor(log2 amax) - 2),
+// 1 BFP4 (E2M1, scale fp16(amax / 6)), 2 MXINT4 (k/4 with |k| <= 7, scale 2^floor(log2 amax)),
+// 3 BINT4 (|k| <= 7, scale fp16(amax / 7)); round to nearest even, saturating.
+// E2M1 codes come from the same conversion instruction as in quantize_group and are decoded again
+// in hardware (e2m1x2 -> f16x2).  With a power-of-two scale the difference is exact in the scaled
+// domain; with an fp16 scale it is one fused multiply-add.  Squares and their sum are fp32.
+__device__ __forceinline__ float group_error(const uint64_t (&P)[16], uint32_t cbits, int format) {
   const float c = __uint_as_float(cbits);
   const uint64_t cc = pack2(c, c);
   float y[32];
 #pragma unroll
-  for (int k = 0; k < 16; ++k) unpack2(mul2(P[k], cc), y[2 * k], y[2 * k + 1]);
+  for (int k = 0; k < 16; ++k) {
+    unpack2(mul2(P[k], cc), y[2 * k], y[2 * k + 1]);
+    y[2 * k] = fabsf(y[2 * k]);             // every format is symmetric: work on magnitudes
+    y[2 * k + 1] = fabsf(y[2 * k + 1]);
+  }
   float m = 0.f;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(y[i]));
+  for (int i = 0; i < 32; ++i) m = fmaxf(m, y[i]);
   const uint32_t ef = __float_as_uint(m) >> 23;
-  const uint32_t s = ef > 2u ? ef - 2u : 0u;
-  const float inv = __uint_as_float((254u - s) << 23);                    // 2^-E, E = s - 127
-  const float pe = __uint_as_float(s >= 1u ? (s << 23) : 0x00400000u);    // 2^E (2^-127 is subnormal)
-  float acc = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; i += 2) {
-    const float r0 = __fmul_rn(y[i], inv), r1 = __fmul_rn(y[i + 1], inv);
+  auto e2m1 = [](float r0, float r1, float& q0, float& q1) {
     uint32_t h;
     asm("{ .reg .b8 b; cvt.rn.satfinite.e2m1x2.f32 b, %2, %1; cvt.rn.f16x2.e2m1x2 %0, b; }" : "=r"(h) : "f"(r0), "f"(r1));
-    const float q0 = __half2float(__ushort_as_half((unsigned short)(h & 0xFFFFu)));
-    const float q1 = __half2float(__ushort_as_half((unsigned short)(h >> 16)));
-    const float d0 = __fsub_rn(r0, q0), d1 = __fsub_rn(r1, q1);
+    q0 = __half2float(__ushort_as_half((unsigned short)(h & 0xFFFFu)));
+    q1 = __half2float(__ushort_as_half((unsigned short)(h >> 16)));
+  };
+  float acc = 0.f;
+  if (format == 0 || format == 2) {
+    const uint32_t s = format == 0 ? (ef > 2u ? ef - 2u : 0u) : ef;
+    const float inv = __uint_as_float((254u - s) << 23);                    // 2^-E, E = s - 127
+    const float pe = __uint_as_float(s >= 1u ? (s << 23) : 0x00400000u);    // 2^E (2^-127 is subnormal)
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+      const float r0 = __fmul_rn(y[i], inv), r1 = __fmul_rn(y[i + 1], inv);
+      float q0, q1;
+      if (format == 0) {
+        e2m1(r0, r1, q0, q1);
+      } else {
+        q0 = 0.25f * (float)min(__float2int_rn(__fmul_rn(r0, 4.f)), 7);
+        q1 = 0.25f * (float)min(__float2int_rn(__fmul_rn(r1, 4.f)), 7);
+      }
+      const float d0 = __fsub_rn(r0, q0), d1 = __fsub_rn(r1, q1);
+      acc = __fadd_rn(acc, __fmul_rn(d0, d0));
+      acc = __fadd_rn(acc, __fmul_rn(d1, d1));
+    }
+    return __fmul_rn(__fmul_rn(__fmul_rn(acc, 0.03125f), pe), pe);
+  }
+  // fp16 scale: the fp32 quotient amax / qmax rounded to nearest-even fp16, saturating
+  float sc;
+  {
+    const float quot = __fdiv_rn(m, format == 1 ? 6.f : 7.f);
+    unsigned short hb;
+    asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(hb) : "f"(quot));
+    sc = __half2float(__ushort_as_half(hb));
+  }
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    float q0 = 0.f, q1 = 0.f;
+    if (sc != 0.f) {
+      const float r0 = __fdiv_rn(y[i], sc), r1 = __fdiv_rn(y[i + 1], sc);
+      if (format == 1) {
+        e2m1(r0, r1, q0, q1);
+      } else {
+        q0 = (float)min(__float2int_rn(r0), 7);
+        q1 = (float)min(__float2int_rn(r1), 7);
+      }
+    }
+    const float d0 = __fmaf_rn(-q0, sc, y[i]), d1 = __fmaf_rn(-q1, sc, y[i + 1]);
     acc = __fadd_rn(acc, __fmul_rn(d0, d0));
     acc = __fadd_rn(acc, __fmul_rn(d1, d1));
   }
-  return __fmul_rn(__fmul_rn(__fmul_rn(acc, 0.03125f), pe), pe);
+  return __fmul_rn(acc, 0.03125f);
 }
 
 // SIGNS: the randomised rotation R_i = diag(s) H / sqrt(block) (paper Sec. 5.1) — the channel signs

@@ -37,6 +37,7 @@ struct Params {
   int chunks_per_row;           // ceil(groups_padded / 32)
   int total_tasks;              // rows_padded * chunks_per_row; one task = one warp, 32 groups of a row
   float* mse;                   // STATS kernels: [M, K/32] per-group quantisation error instead of codes/scales
+  int format;                   // STATS kernels: which 4-bit format (see rq::group_error)
 };
 
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(con
     const int g = chunk * 32 + lane;
     const bool live = row < p.M && g < ng;
     if (STATS) {
-      const float e = rq::group_error(P, cbits);
+      const float e = rq::group_error(P, cbits, p.format);
       if (live) p.mse[(int64_t)row * ng + g] = e;
 #pragma unroll
       for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
@@ -184,6 +185,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int l
   p.layout = (int)layout;
   p.signs = static_cast<const uint16_t*>(signs);
   p.mse = nullptr;
+  p.format = 0;
   p.rows_padded = (int)(layout == BRO_LAYOUT_GEMM ? (M + 127) / 128 * 128 : M);
   p.groups_padded = (int)(layout == BRO_LAYOUT_GEMM ? scale_kblocks * 4 : K / 32);
   p.chunks_per_row = (p.groups_padded + 31) / 32;
@@ -193,7 +195,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int l
 
 // Per-group quantisation error only: mse[M, K/32] (fp32).
 inline bro_status launch_stats(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs,
-                               float* mse, int sm_count, cudaStream_t st) {
+                               int format, float* mse, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M; p.K = K; p.ldx = ldx;
@@ -203,6 +205,7 @@ inline bro_status launch_stats(const void* x, int64_t M, int64_t K, int64_t ldx,
   p.layout = (int)BRO_LAYOUT_CANONICAL;
   p.signs = static_cast<const uint16_t*>(signs);
   p.mse = mse;
+  p.format = format;
   p.rows_padded = (int)M;
   p.groups_padded = (int)(K / 32);
   p.chunks_per_row = (p.groups_padded + 31) / 32;

@@ -28,6 +28,7 @@ struct Params {
   int rows_per_iter;     // blockDim.x / threads_per_row
   const uint16_t* signs; // [K] bf16 +-1 for the randomised rotation diag(s) H / sqrt(K), or nullptr
   float* mse;            // if set: write the per-group quantisation error [M, K/32] instead of codes/scales
+  int format;            // ... for this 4-bit format (see rq::group_error)
 };
 
 template <int kMaxThreads>
@@ -94,7 +95,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
       }
     }
     if (p.mse) {                 // analysis mode (uniform over the grid)
-      const float e = rq::group_error(P, cbits);
+      const float e = rq::group_error(P, cbits, p.format);
       if (live) p.mse[row * (p.K >> 5) + gi] = e;
       continue;
     }
@@ -115,7 +116,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
 }
 
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
-                         void* scales, float* mse, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+                         void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M;
@@ -127,6 +128,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   p.layout = (int)layout;
   p.signs = static_cast<const uint16_t*>(signs);
   p.mse = mse;
+  p.format = format;
   int lg = 0;
   while (((int64_t)1 << lg) < K) ++lg;
   p.log2k = lg;

@@ -18,17 +18,19 @@ def bro():
     return binding
 
 
-def reference(x, block, signs=None):
+def reference(x, block, signs=None, fmt="mxfp4"):
     sb = None if signs is None else synth.bf16_bits(signs)
     y = oracle.rotate(synth.bf16_bits(x), block, sb)
+    if fmt != "mxfp4":
+        return oracle.group_error(y, fmt)
     codes, scales = oracle.quantize(y)
     return oracle.group_mse(y, codes, scales)
 
 
-def gpu(bro, x, block, signs=None):
+def gpu(bro, x, block, signs=None, fmt="mxfp4"):
     M, K = x.shape
     mse = torch.full((M, K // 32), float("nan"), dtype=torch.float32, device="cuda")
-    bro.group_quant_error(x.cuda(), block, mse, None if signs is None else signs.cuda())
+    bro.group_quant_error(x.cuda(), block, mse, None if signs is None else signs.cuda(), fmt=fmt)
     assert bro.last_device_status() == 0
     return mse.cpu().numpy().astype(np.float64)
 
@@ -73,3 +75,30 @@ def test_block_sweep_ordering_on_outlier_channels(bro):
     x = synth.activations(512, 4096, seed=4000, recipe=synth.CFG4_RECIPE)
     med = {b: float(np.median(gpu(bro, x, b))) for b in (32, 128, 0)}
     assert med[32] < med[128] < med[0]
+
+
+@pytest.mark.parametrize("fmt", ["bfp4", "mxint4", "bint4"])
+@pytest.mark.parametrize("block", [32, 128, 0])
+def test_comparison_formats_match_the_oracle(bro, fmt, block):
+    """BFP4 / MXINT4 / BINT4 (Sec. 3.1, Fig. 2-3).  With an fp16 scale the difference y - q*s is one
+    fused multiply-add instead of an exact subtraction, still far inside the 1e-5 bar."""
+    x = synth.activations(200, 1024, seed=90)
+    check(gpu(bro, x, block, fmt=fmt), reference(x, block, fmt=fmt))
+    xs = synth.activations(33, 416, seed=91) if block == 32 else None
+    if xs is not None:
+        signs = synth.rotation_signs(416, seed=92)
+        check(gpu(bro, xs, 32, signs, fmt=fmt), reference(xs, 32, signs, fmt=fmt))
+
+
+def test_formats_on_degenerate_rows(bro):
+    """Zero rows, tiny rows (fp16 scale underflows to zero: everything quantises to zero) and huge
+    rows (fp16 scale saturates at 65504)."""
+    K = 128
+    x = torch.zeros((4, K), dtype=torch.bfloat16)
+    g = torch.Generator().manual_seed(1)
+    base = torch.randn(K, generator=g)
+    x[1] = (base * 2.0 ** -30).to(torch.bfloat16)
+    x[2] = (base * 2.0 ** 20).to(torch.bfloat16)
+    x[3] = base.to(torch.bfloat16)
+    for fmt in ("bfp4", "mxint4", "bint4"):
+        check(gpu(bro, x, 32, fmt=fmt), reference(x, 32, fmt=fmt))
