@@ -38,6 +38,7 @@ constexpr int kBK = 256;                    // elements per K step = 128 bytes o
 constexpr int kThreads = 192;
 constexpr int kATileBytes = kBM * 128;      // 16 KiB
 constexpr int kChunkCols = 32;              // epilogue chunk: 32 fp32 columns per tcgen05.ld
+constexpr int kRasterRows = 8;              // tile rows per raster band
 constexpr int kStageOutBytes = kBM * kChunkCols * 2;   // 8 KiB bf16 staging per chunk
 
 template <int BN> struct Cfg {
@@ -234,7 +235,15 @@ __device__ __forceinline__ void decode_unit(const Params& p, int u, int& m0, int
     half = idx & 1;
     bn = BN / 2;
   }
-  const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+  // Tile order: bands of kRasterRows tile rows, column by column inside a band, so that the CTAs
+  // running at the same time share a few activation panels and a few weight panels (with plain
+  // row-major order and a weight matrix larger than L2, every tile row streams W from HBM again).
+  const int per_band = kRasterRows * p.tiles_n;
+  const int band = tile / per_band;
+  const int within = tile - band * per_band;
+  const int rows = min(kRasterRows, p.tiles_m - band * kRasterRows);
+  const int tn = within / rows;
+  const int tm = band * kRasterRows + (within - tn * rows);
   m0 = tm * kBM;
   n0 = tn * BN + half * (BN / 2);
 }
