@@ -354,8 +354,12 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
 template <int CHUNKS, bool OVERLAP, bool OUT_F32, typename ReleaseShared, typename ReleaseAll>
 __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int lane, int row0, int n0, int64_t M,
                                               int64_t N, void* y, int64_t ldy, const CUtensorMap* tmy,
-                                              uint32_t stage_buf, ReleaseShared release_shared,
-                                              ReleaseAll release_all) {
+                                              uint32_t stage_buf, uint32_t stage_stride,
+                                              ReleaseShared release_shared, ReleaseAll release_all) {
+  // stage_stride == 0: one staging buffer, reused pair after pair (each reuse waits until the
+  // previous TMA store has read it).  stage_stride != 0: pair i has its own buffer at
+  // stage_buf + i * stage_stride and nothing waits — used for a CTA's final tile, whose epilogue
+  // is the kernel's tail and for which the idle operand stages provide the room.
   static_assert(CHUNKS % 2 == 0, "chunks are processed in pairs");
   constexpr int PAIRS = CHUNKS / 2;
   const int64_t row = (int64_t)row0 + lane;
@@ -383,7 +387,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
       }
     }
   };
-  auto emit = [&](const uint32_t (&r0)[32], const uint32_t (&r1)[32], int pr) {
+  auto emit = [&](const uint32_t (&r0)[32], const uint32_t (&r1)[32], int pr, int pi) {
     const int col0 = n0 + pr * 2 * kChunkCols;
     if (OUT_F32) {
       store_f32(r0, col0);
@@ -395,11 +399,12 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[j]) : "f"(__uint_as_float(r0[2 * j + 1])), "f"(__uint_as_float(r0[2 * j])));
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[16 + j]) : "f"(__uint_as_float(r1[2 * j + 1])), "f"(__uint_as_float(r1[2 * j])));
       }
+      const uint32_t sbuf = stage_buf + (uint32_t)pi * stage_stride;
       // the TMA store that last read the staging buffer must be done reading it
-      bulk_wait_read_if<0>(issue);
+      if (stage_stride == 0u) bulk_wait_read_if<0>(issue);
       __syncwarp();
       // row `lane` of the box: 128 bytes, 16-byte pieces XOR-swizzled with lane & 7
-      const uint32_t rowaddr = stage_buf + (uint32_t)lane * 128u;
+      const uint32_t rowaddr = sbuf + (uint32_t)lane * 128u;
       const uint32_t sw = (uint32_t)lane & 7u;
 #pragma unroll
       for (int j = 0; j < 8; ++j) sts128(rowaddr + ((j ^ sw) << 4), h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
@@ -408,7 +413,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
       // A TMA store clips at 16-byte granularity: when N is not a multiple of 8 the ragged last
       // pair is written from registers instead, element by element.
       const bool ragged = ((N & 7) != 0) && ((int64_t)col0 + 2 * kChunkCols > N);
-      tma_store_2d_if((col0 < N && row0 < M && !ragged) ? issue : 0u, tmy, stage_buf, col0, row0);
+      tma_store_2d_if((col0 < N && row0 < M && !ragged) ? issue : 0u, tmy, sbuf, col0, row0);
       bulk_commit_if(issue);           // (possibly empty) keeps the group count in step
       if (ragged && row < M) {
         uint16_t* dst = static_cast<uint16_t*>(y) + row * ldy + col0;
@@ -429,7 +434,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
       tc_ld32(tmem_acc + pair_of(pi + 1) * 2 * kChunkCols + kChunkCols, rd);
     }
     released(pi);
-    emit(ra, rb, pair_of(pi));
+    emit(ra, rb, pair_of(pi), pi);
     if (pi + 1 < PAIRS) {
       tc_wait_ld();
       if (pi + 2 < PAIRS) {
@@ -437,7 +442,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int buf, int la
         tc_ld32(tmem_acc + pair_of(pi + 2) * 2 * kChunkCols + kChunkCols, rb);
       }
       released(pi + 1);
-      emit(rc, rd, pair_of(pi + 1));
+      emit(rc, rd, pair_of(pi + 1), pi + 1);
     }
   }
 }
@@ -582,15 +587,18 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
       if (!mbar_wait_warp(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL)) break;
       tc_fence_after();
       const uint32_t tmem_acc = tmem_base + buf * C::kAccStride + ((uint32_t)(q * 32) << 16);
-      const uint32_t stage_buf = sOut + (uint32_t)q * (32u * 128u);
+      // the final tile of this CTA stages every pair in its own 4 KiB of the (now idle) A stages
+      const bool last = u + (int)gridDim.x >= p.total_units;
+      const uint32_t stage_buf = last ? sA + (uint32_t)q * (4u * 4096u) : sOut + (uint32_t)q * (32u * 128u);
+      const uint32_t stage_stride = last ? 4096u : 0u;
       auto release_shared = [&] { mbar_arrive(bar_ovl_free + 8 * buf); };
       auto release_all = [&] { mbar_arrive(bar_acc_free + 8 * buf); };
       if (bn == BN)
         epilogue_tile<C::kChunks, C::kOverlap, OUT_F32>(tmem_acc, buf, lane, m0 + q * 32, n0, p.M, p.N, p.y, p.ldy, &tmy,
-                                                        stage_buf, release_shared, release_all);
+                                                        stage_buf, stage_stride, release_shared, release_all);
       else
         epilogue_tile<C::kChunks / 2, C::kOverlap, OUT_F32>(tmem_acc, buf, lane, m0 + q * 32, n0, p.M, p.N, p.y, p.ldy,
-                                                            &tmy, stage_buf, release_shared, release_all);
+                                                            &tmy, stage_buf, stage_stride, release_shared, release_all);
     }
     // the staging buffer must have been read before this CTA's shared memory goes away; the writes
     // themselves complete with the kernel

@@ -222,7 +222,7 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
       const uint32_t acc_free_leader = map_to_cta(bar_acc_free + 8 * buf, 0);
       gemm::epilogue_tile<kChunks, true, OUT_F32>(
           tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16), buf, lane, tm * 256 + (int)rank * kBM + q * 32,
-          tn * kBN, p.M, p.N, p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u),
+          tn * kBN, p.M, p.N, p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u), 0u,
           [&] { mbar_arrive_cluster(ovl_free_leader); }, [&] { mbar_arrive_cluster(acc_free_leader); });
     }
     // the staging buffer must have been read before this CTA's shared memory goes away; the writes
