@@ -68,6 +68,7 @@ struct Params {
   // tile count leaves the last round of the grid less than half full, the remaining tiles are cut
   // into two 128 x BN/2 halves each (units full_units ..), so that the last round keeps every SM busy.
   int full_units, total_units;
+  int a_box_bytes;          // bytes one activation TMA box brings (fewer than 128 rows when M is small)
   int w_static;             // the weight operand was complete before the previous kernel started (see launch)
 };
 
@@ -521,7 +522,7 @@ gemm_mxfp4_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant
         const int nblk_valid = (int64_t)n0 >= p.N ? 0 : ((bn == 256 && (int64_t)n0 + 128 < p.N) ? 2 : 1);
         const uint32_t full = bar_full + 8 * st;
         if (part & 1) {
-          mbar_arrive_expect_tx(full, kATileBytes + bn * 128 + C::kSfaBytes + nblk_valid * 1024);
+          mbar_arrive_expect_tx(full, p.a_box_bytes + bn * 128 + C::kSfaBytes + nblk_valid * 1024);
           tma_load_2d(sB + st * C::kBTileBytes, bn == BN ? &tmw : &tmw_half, ks * 128, n0, full);
           const uint8_t* sfb_src = p.wscales + (int64_t)(n0 / 128) * p.kblocks * 512;
           for (int nb = 0; nb < nblk_valid; ++nb)
@@ -668,7 +669,13 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   p.kblocks = 2 * (int64_t)p.num_k_steps;
   p.w_static = w_static ? 1 : 0;
   CUtensorMap tma, tmw, tmy;
-  bro_status rc = make_codes_map(&tma, acodes, M, K, kBM);
+  // With fewer than 128 tokens the activation box covers only the next power of two of rows (at
+  // least 8): rows the box does not bring keep whatever the shared-memory stage held — finite fp4
+  // codes under zero-padded scales — and feed output rows that are never stored.
+  int a_rows = kBM;
+  while (a_rows > 8 && a_rows / 2 >= M) a_rows /= 2;
+  p.a_box_bytes = a_rows * 128;
+  bro_status rc = make_codes_map(&tma, acodes, M, K, a_rows);
   if (rc != BRO_OK) return rc;
   rc = make_codes_map(&tmw, wcodes, N, K, bn);
   if (rc != BRO_OK) return rc;
