@@ -43,7 +43,7 @@ struct Params {
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
 // (rq::group_error) — the analysis behind the paper's regular-block / outlier-block comparison.
 template <int LOG2B, bool SIGNS, bool STATS>
-__global__ void __launch_bounds__(kThreads, 2) rotate_quantize_direct_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, 3) rotate_quantize_direct_kernel(const Params p) {
   const int lane = threadIdx.x & 31;
   const int num_warps = (int)gridDim.x * kWarps;
   const int ng = (int)(p.K >> 5);
