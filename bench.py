@@ -55,10 +55,14 @@ def select_shapes(args):
 # one value per shape).  The figures belong to one exact version of the kernels: `sources` is the SHA-256
 # over the files of csrc/ at capture time, and the benchmark reports null when they have changed since.
 # (The outputs of these shapes, 8-33 MB, are still dirty in the 126 MB L2 when the kernel ends, which is
-# why the traffic is below the algorithmic bytes.)
+# why the traffic is below the algorithmic bytes.)  "cfg3" holds the one shape captured with `--set full
+# -k regex:gemm_mxfp4 -s 3 -c 2` under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel
+# captured with `-k regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
 NCU_TRAFFIC = {
     "sources": "f463f961fffcca8816458e481e02ff2881f39cf7104610b8320a91e4226e0985",
     "cfg2": {(2048, 2048, 2048): 4537088, (2048, 2048, 8192): 11223040, (2048, 8192, 2048): 17906432},
+    "cfg3": {(4096, 4096, 14336): 117767680},
+    "cfg4": {(16384, 4096, 32): 153049344},
 }
 
 
@@ -599,7 +603,8 @@ def run_rotate_quantize_only(args):
            "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse, "gpu_format_study": format_study,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                        "traffic": None, "algorithmic_bytes": bytes_per_launch,
+                        "traffic": ncu_traffic("cfg4", [(M, K, blocks[0] if blocks[0] else K)]),
+                        "algorithmic_bytes": bytes_per_launch,
                         "timing": f"CUDA events around groups of {group} back-to-back launches, {n_groups} groups per size"}}
     print(json.dumps(out), flush=True)
 
