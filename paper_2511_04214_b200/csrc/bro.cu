@@ -459,8 +459,10 @@ bro_status bro_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t l
   unsigned char* gws = ascales + scales_sz;
   bro_status rc = bro_rotate_quantize_mxfp4(x_bf16, M, K, ldx, block, acodes, ascales, BRO_LAYOUT_GEMM, stream);
   if (rc != BRO_OK) return rc;
-  return bro_gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16,
-                        gemm_sz ? gws : nullptr, gemm_sz, stream);
+  // (as in bro_linear: the packed weights are older than the kernel just enqueued, so the GEMM may
+  // fetch its first weight tiles before that kernel has finished)
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gemm_sz ? gws : nullptr,
+                   gemm_sz, stream, true);
 }
 
 }  // extern "C"
