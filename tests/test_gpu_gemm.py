@@ -248,3 +248,35 @@ def test_config2_shape_sampled(bro):
     y_ref, S = oracle.gemm_mxfp4_points(ac, asc, wc, wsc, pm, pn)
     got = y[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()].cpu().numpy().astype(np.float64)
     assert np.all(np.abs(got - y_ref) <= 1e-5 * S + 1e-6)
+
+
+def test_whole_layer_is_deterministic_and_graph_safe(bro):
+    """Same inputs -> same bits, call after call and when replayed from a CUDA graph (no atomics, a
+    fixed order of tensor-core operations, no allocation or synchronisation inside the calls)."""
+    M, K, N = 300, 1024, 776
+    x = synth.activations(M, K, seed=77).cuda()
+    w = synth.weights(N, K, seed=78).cuda()
+    wcodes = bro.alloc_codes(N, K)
+    wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM)
+    bro.pack_weights(w, 32, wcodes, wscales)
+    ws = bro.alloc_workspace(bro.linear_workspace_bytes(M, N, K))
+    y1 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    bro.linear(x, 32, wcodes, wscales, N, y1, ws)
+    bro.linear(x, 32, wcodes, wscales, N, y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+    y3 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        bro.linear(x, 32, wcodes, wscales, N, y3, ws, stream=s)        # warm-up outside capture
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            bro.linear(x, 32, wcodes, wscales, N, y3, ws, stream=s)
+        y3.fill_(float("nan"))
+        g.replay()
+        g.replay()
+    torch.cuda.synchronize()
+    assert bro.last_device_status() == 0
+    assert torch.equal(y1.view(torch.int16), y3.view(torch.int16))
