@@ -59,10 +59,10 @@ def select_shapes(args):
 # -k regex:gemm_mxfp4 -s 3 -c 2` under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel
 # captured with `-k regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
 NCU_TRAFFIC = {
-    "sources": "ceb0cb21a0fda3bb5cf9b1faf5e487bbf894b99a70c1dbf0e6b335c24f702da7",
-    "cfg2": {(2048, 2048, 2048): 4536832, (2048, 2048, 8192): 11226624, (2048, 8192, 2048): 17908224},
-    "cfg3": {(4096, 4096, 14336): 117767680},
-    "cfg4": {(16384, 4096, 32): 153049344},
+    "sources": "a56c7b2c27f9fda55cb57728994f0f09dec376166defeab029151a2e894eba40",
+    "cfg2": {(2048, 2048, 2048): 4537344, (2048, 2048, 8192): 11223040, (2048, 8192, 2048): 17906944},
+    "cfg3": {(4096, 4096, 14336): 113546752},
+    "cfg4": {(16384, 4096, 32): 152742400},
 }
 
 

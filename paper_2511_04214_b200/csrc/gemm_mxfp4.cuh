@@ -38,7 +38,7 @@ constexpr int kBK = 256;                    // elements per K step = 128 bytes o
 constexpr int kThreads = 192;
 constexpr int kATileBytes = kBM * 128;      // 16 KiB
 constexpr int kChunkCols = 32;              // epilogue chunk: 32 fp32 columns per tcgen05.ld
-constexpr int kRasterRows = 8;              // tile rows per raster band
+constexpr int kRasterRows = 8;              // tile rows per raster band (12 when the weights do not fit L2, see launch_tile)
 constexpr int kStageOutBytes = kBM * kChunkCols * 2;   // 8 KiB bf16 staging per chunk
 
 template <int BN> struct Cfg {
@@ -68,6 +68,7 @@ struct Params {
   // tile count leaves the last round of the grid less than half full, the remaining tiles are cut
   // into two 128 x BN/2 halves each (units full_units ..), so that the last round keeps every SM busy.
   int full_units, total_units;
+  int raster_rows;          // tile rows per raster band
   int a_box_bytes;          // bytes one activation TMA box brings (fewer than 128 rows when M is small)
   int w_static;             // the weight operand was complete before the previous kernel started (see launch)
 };
@@ -236,15 +237,15 @@ __device__ __forceinline__ void decode_unit(const Params& p, int u, int& m0, int
     half = idx & 1;
     bn = BN / 2;
   }
-  // Tile order: bands of kRasterRows tile rows, column by column inside a band, so that the CTAs
+  // Tile order: bands of raster_rows tile rows, column by column inside a band, so that the CTAs
   // running at the same time share a few activation panels and a few weight panels (with plain
   // row-major order and a weight matrix larger than L2, every tile row streams W from HBM again).
-  const int per_band = kRasterRows * p.tiles_n;
+  const int per_band = p.raster_rows * p.tiles_n;
   const int band = tile / per_band;
   const int within = tile - band * per_band;
-  const int rows = min(kRasterRows, p.tiles_m - band * kRasterRows);
+  const int rows = min(p.raster_rows, p.tiles_m - band * p.raster_rows);
   const int tn = within / rows;
-  const int tm = band * kRasterRows + (within - tn * rows);
+  const int tm = band * p.raster_rows + (within - tn * rows);
   m0 = tm * kBM;
   n0 = tn * BN + half * (BN / 2);
 }
@@ -624,6 +625,11 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
   if (total > 0x3FFFFFFF) return BRO_ERR_UNSUPPORTED;
   p.total_tiles = (int)total;
+  // One wave of CTAs covers raster_rows activation panels and sm_count / raster_rows weight panels.
+  // 8 rows is best while the packed weights stay in L2 between bands; when they do not (measured
+  // with 125 MB of weights: 2.7 % faster at M = 32768), the squarer 12 x 12 wave re-reads fewer
+  // weight bytes from HBM.
+  p.raster_rows = (double)p.N * (double)p.K * (17.0 / 32.0) > 64.0 * 1024 * 1024 ? 12 : kRasterRows;
   // Rounds of the persistent grid: when the last round would leave at least half of the SMs idle,
   // its tiles are cut into two half-width units each (BRO_GEMM_SPLIT=0 switches this off).
   int64_t grid = total < sm_count ? total : sm_count;
