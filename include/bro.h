@@ -19,9 +19,17 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
  *     enqueue work and return without synchronising.  The returned status covers argument
  *     validation and launch errors only.
- *   - Every device-side wait is bounded.  If one expires (which indicates a bug or a broken
- *     device, never a data condition) the kernel records BRO_ERR_TIMEOUT in a device-side
- *     status word and returns; bro_last_device_status() reads and clears that word.
+ *   - Every device-side wait is bounded by a time budget (two seconds on the device's own
+ *     nanosecond timer).  If one expires (which indicates a bug or a broken device, never a data
+ *     condition) the kernel records BRO_ERR_TIMEOUT and the place of the wait in a device-side
+ *     status word and returns; bro_last_device_status() reads and clears that word.  There is ONE
+ *     status word per device, shared by all streams and all calls on that device (it lives in the
+ *     library's device image, not in a caller buffer, so that entry points without a workspace
+ *     can report too): it says that some kernel since the last read gave up, not which call.
+ *   - The library keeps no other state that affects results: which kernel variant runs is a
+ *     function of the arguments alone (the *_ex entry points take explicit flags; nothing is
+ *     read from the environment).  One-time per-device set-up (kernel attributes) is
+ *     thread-safe.
  *   - No exception crosses this boundary.  Invalid arguments return an error code; they never
  *     lead to undefined behaviour.  M == 0 or N == 0 returns BRO_OK without a launch.
  *   - bf16 tensors are row-major with a leading dimension in ELEMENTS.
@@ -89,6 +97,10 @@ size_t bro_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * device: BRO_OK, or BRO_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last call.
  * BRO_ERR_CUDA if the synchronisation itself reports an error. */
 bro_status bro_last_device_status(void* stream);
+/* The same, and *site (if not NULL) receives the number of the wait that expired (0 if none):
+ * 1-3 rotate+quantize ring (full / empty / drain), 4-9 GEMM (operands full / stage empty /
+ * accumulator full / accumulator free / drain / tensor memory), 10 the self-test below. */
+bro_status bro_last_device_status_ex(void* stream, int* site);
 
 /*
  * Online activation path (Sec. 4.3 Eq. 1 + Sec. 4.1): for every row of x[M, K] (bf16) and every
@@ -189,6 +201,41 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
                                      void* stream);
 
 /*
+ * ---- tuning and testing -------------------------------------------------------------------------
+ * The *_ex entry points are the plain ones plus a `flags` word that forces a kernel variant the
+ * library would not pick by itself for this problem (the plain entry points pass 0).  Every variant
+ * computes the same function: codes and scales are bit-identical, GEMM results agree within the
+ * accumulation-order tolerance.  They exist so that each variant can be tested and timed on any
+ * shape; `signs_bf16` may be NULL (plain rotation) or the +-1 vector of the randomised rotation.
+ */
+#define BRO_FLAG_RQ_TMA_RING 0x1u     /* rotate+quantize: shared-memory ring fed by TMA (block 32/64/128) */
+#define BRO_FLAG_RQ_DIRECT 0x2u       /* rotate+quantize: register-streaming kernel (block 32/64/128) */
+#define BRO_FLAG_GEMM_PAIR 0x10u      /* GEMM: two CTAs per 256 x 256 tile (cta_group::2) */
+#define BRO_FLAG_GEMM_TILE_N128 0x20u /* GEMM: 128 x 128 tiles */
+#define BRO_FLAG_GEMM_TILE_N256 0x40u /* GEMM: 128 x 256 tiles even when N <= 128 */
+#define BRO_FLAG_GEMM_NO_SPLIT 0x80u  /* GEMM: no half-width units in the last round, no K split */
+bro_status bro_rotate_quantize_mxfp4_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                        const void* signs_bf16, void* codes, void* scales,
+                                        bro_layout layout, uint32_t flags, void* stream);
+bro_status bro_gemm_mxfp4_ex(const void* acodes, const void* ascales, const void* wcodes,
+                             const void* wscales, int64_t M, int64_t N, int64_t K, void* y, int64_t ldy,
+                             bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
+                             uint32_t flags, void* stream);
+bro_status bro_linear_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                         const void* signs_bf16, const void* wcodes, const void* wscales, int64_t N,
+                         void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                         uint32_t flags, void* stream);
+
+/*
+ * Self-test of the bounded-wait machinery (no counterpart in the paper): launches one warp that
+ * waits, with a budget of `budget_ns` nanoseconds (clamped to [1 us, 100 ms]), on a barrier that
+ * nothing ever completes.  The wait runs out, the warp records BRO_ERR_TIMEOUT with site 10 in the
+ * device status word and the kernel ends normally — nothing faults, and the context stays usable.
+ * A following bro_last_device_status() therefore returns BRO_ERR_TIMEOUT once, then BRO_OK.
+ */
+bro_status bro_selftest_expire_wait(uint64_t budget_ns, void* stream);
+
+/*
  * bro_linear for a caller whose activations and result live in HOST memory (pinned memory gives
  * asynchronous copies).  Copies x_host[M, K] (dense, ldx = K) to the device staging buffer,
  * runs bro_linear, and copies y[M, N] (dense) back to y_host, all on `stream`.
@@ -220,9 +267,12 @@ bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int bl
  * bro_last_cuda_error().  All other arguments, requirements and errors are those of bro_linear.
  *
  * Set-up: the first call on each device looks up the array's device address (the name the
- * host code sees is only a handle, not an address a kernel could use) and opts the kernels in to
- * their shared-memory sizes.  Make that first call with the device current and outside any
- * stream capture.
+ * host code sees is only a handle, not an address a kernel could use).  Make that first call with
+ * the device current and outside any stream capture.  Separately, as for every entry point of
+ * this library, the first launch of each kernel variant on a device (one per block size, per
+ * size class of the input, per GEMM tile width and output type) loads that kernel and opts it in
+ * to its shared-memory size: run one call of every (block, shape class) you will use before
+ * capturing.  With block = 0 the call also enqueues a memset of the scale buffer's padding.
  *
  * Sharing: every call on a device uses the same array and finds in it whatever the previous
  * call left.  Each call rewrites everything it later reads (padding included), so stale contents

@@ -26,7 +26,17 @@ EXPORTS = [
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host", "bro_linear_static",
     "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt",
+    "bro_last_device_status_ex", "bro_selftest_expire_wait",
+    "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
 ]
+
+# kernel-selection flags of the *_ex entry points (testing and tuning)
+FLAG_RQ_TMA_RING = 0x1
+FLAG_RQ_DIRECT = 0x2
+FLAG_GEMM_PAIR = 0x10
+FLAG_GEMM_TILE_N128 = 0x20
+FLAG_GEMM_TILE_N256 = 0x40
+FLAG_GEMM_NO_SPLIT = 0x80
 
 
 class BroError(RuntimeError):
@@ -42,7 +52,8 @@ def _load() -> ctypes.CDLL:
             f"{_SO} is missing: build it with `python -m paper_2511_04214_b200.build` "
             "(there is no fallback path)")
     L = ctypes.CDLL(_SO)
-    i64, p, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    i64, p, ci, sz, u32, u64 = (ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint32,
+                                ctypes.c_uint64)
     L.bro_status_string.restype = ctypes.c_char_p
     L.bro_status_string.argtypes = [ci]
     L.bro_last_cuda_error.restype = ctypes.c_char_p
@@ -81,6 +92,16 @@ def _load() -> ctypes.CDLL:
     L.bro_group_quant_error_fmt.argtypes = [p, i64, i64, i64, ci, p, ci, p, p]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
+    L.bro_last_device_status_ex.restype = ci
+    L.bro_last_device_status_ex.argtypes = [p, ctypes.POINTER(ci)]
+    L.bro_selftest_expire_wait.restype = ci
+    L.bro_selftest_expire_wait.argtypes = [u64, p]
+    L.bro_rotate_quantize_mxfp4_ex.restype = ci
+    L.bro_rotate_quantize_mxfp4_ex.argtypes = [p, i64, i64, i64, ci, p, p, p, ci, u32, p]
+    L.bro_gemm_mxfp4_ex.restype = ci
+    L.bro_gemm_mxfp4_ex.argtypes = [p, p, p, p, i64, i64, i64, p, i64, ci, p, sz, u32, p]
+    L.bro_linear_ex.restype = ci
+    L.bro_linear_ex.argtypes = [p, i64, i64, i64, ci, p, p, p, i64, p, i64, p, sz, u32, p]
     return L
 
 
@@ -130,6 +151,18 @@ def last_device_status(stream=None) -> int:
     return int(lib.bro_last_device_status(_stream(stream)))
 
 
+def last_device_status_ex(stream=None):
+    """(status, site): the device status word of the current device, read and cleared."""
+    site = ctypes.c_int(0)
+    code = int(lib.bro_last_device_status_ex(_stream(stream), ctypes.byref(site)))
+    return code, int(site.value)
+
+
+def selftest_expire_wait(budget_ns: int = 1_000_000, stream=None) -> None:
+    """Launch the one-warp self-test whose bounded wait runs out (see include/bro.h)."""
+    _check(lib.bro_selftest_expire_wait(int(budget_ns), _stream(stream)), "bro_selftest_expire_wait")
+
+
 def alloc_codes(rows: int, K: int, device="cuda") -> torch.Tensor:
     return torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
 
@@ -146,9 +179,14 @@ def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
 
 
 def rotate_quantize_mxfp4(x: torch.Tensor, block: int, codes: torch.Tensor, scales: torch.Tensor,
-                          layout: int = LAYOUT_GEMM, stream=None) -> None:
+                          layout: int = LAYOUT_GEMM, stream=None, flags: int = 0, signs=None) -> None:
     assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
     M, K = x.shape
+    if flags or signs is not None:
+        _check(lib.bro_rotate_quantize_mxfp4_ex(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K), block,
+                                                _ptr(signs), _ptr(codes), _ptr(scales), layout, flags,
+                                                _stream(stream)), "bro_rotate_quantize_mxfp4_ex")
+        return
     _check(lib.bro_rotate_quantize_mxfp4(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K),
                                          block, _ptr(codes), _ptr(scales), layout, _stream(stream)),
            "bro_rotate_quantize_mxfp4")
@@ -163,19 +201,31 @@ def pack_weights(w: torch.Tensor, block: int, wcodes: torch.Tensor, wscales: tor
 
 
 def gemm_mxfp4(acodes, ascales, wcodes, wscales, M: int, N: int, K: int, y: torch.Tensor,
-               workspace=None, stream=None) -> None:
+               workspace=None, stream=None, flags: int = 0) -> None:
     out = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
     assert y.dtype in (torch.bfloat16, torch.float32) and y.stride(1) == 1
     wsb = 0 if workspace is None else workspace.numel()
+    if flags:
+        _check(lib.bro_gemm_mxfp4_ex(_ptr(acodes), _ptr(ascales), _ptr(wcodes), _ptr(wscales), M, N, K,
+                                     _ptr(y), y.stride(0) if M > 1 else max(y.stride(0), N), out,
+                                     _ptr(workspace), wsb, flags, _stream(stream)), "bro_gemm_mxfp4_ex")
+        return
     _check(lib.bro_gemm_mxfp4(_ptr(acodes), _ptr(ascales), _ptr(wcodes), _ptr(wscales), M, N, K,
                               _ptr(y), y.stride(0) if M > 1 else max(y.stride(0), N), out,
                               _ptr(workspace), wsb, _stream(stream)), "bro_gemm_mxfp4")
 
 
 def linear(x: torch.Tensor, block: int, wcodes, wscales, N: int, y: torch.Tensor,
-           workspace: torch.Tensor, stream=None) -> None:
+           workspace: torch.Tensor, stream=None, flags: int = 0, signs=None) -> None:
     assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
     M, K = x.shape
+    if flags:
+        _check(lib.bro_linear_ex(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K), block, _ptr(signs),
+                                 _ptr(wcodes), _ptr(wscales), N, _ptr(y),
+                                 y.stride(0) if M > 1 else max(y.stride(0), N), _ptr(workspace),
+                                 workspace.numel(), flags, _stream(stream)), "bro_linear_ex")
+        return
+    assert signs is None, "use linear_rs (or pass flags) for the randomised rotation"
     _check(lib.bro_linear(_ptr(x), M, K, x.stride(0) if M > 1 else max(x.stride(0), K), block,
                           _ptr(wcodes), _ptr(wscales), N, _ptr(y),
                           y.stride(0) if M > 1 else max(y.stride(0), N), _ptr(workspace),

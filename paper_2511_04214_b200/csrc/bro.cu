@@ -125,10 +125,23 @@ bro_status bro::gemm2::make_scale_map(CUtensorMap* map, const void* scales, int6
 
 namespace {
 
+// One warp waits on a barrier that nothing completes: the bounded wait runs out, records its site and
+// the kernel returns normally (see bro_selftest_expire_wait).
+__global__ void expire_wait_kernel(uint64_t budget_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = bro::smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    bro::mbar_init(b, 1);
+    bro::mbar_fence_init();
+  }
+  __syncwarp();
+  bro::mbar_wait(b, 0u, bro::SITE_SELF_TEST, budget_ns);
+}
+
 // ---- rotate + quantise ---------------------------------------------------------------------------
 bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, int block,
                                   const void* signs, void* codes, void* scales, bro_layout layout,
-                                  cudaStream_t st) {
+                                  uint32_t flags, cudaStream_t st) {
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (M == 0 && (layout == BRO_LAYOUT_CANONICAL || layout == BRO_LAYOUT_GEMM)) return BRO_OK;
@@ -149,12 +162,14 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
     return bro::rqg::launch(x, M, K, ldx, signs, codes, scales, nullptr, 0, layout, gemm_scale_kblocks(K), di.sm_count, st);
   }
 
-  // Register-streaming kernel by default; BRO_RQ_TMA=1 selects the TMA-ring kernel (also used when
-  // the task index would not fit 31 bits).
-  // (it wins for block 32 at every size and for small inputs; for blocks of 64 / 128 on large
-  // inputs its extra registers cost occupancy and the TMA ring is faster)
-  bool direct = bro::rqd::supports(M, K, layout, gemm_scale_kblocks(K)) && (B == 32 || M * K <= ((int64_t)1 << 23));
-  if (const char* e = getenv("BRO_RQ_TMA")) direct = direct && atoi(e) == 0;
+  // Register-streaming kernel by default (the TMA-ring kernel when the task index would not fit
+  // 31 bits): it wins for block 32 at every size and for small inputs; for blocks of 64 / 128 on
+  // large inputs its extra registers cost occupancy and the TMA ring is faster.  The flags of the
+  // *_ex entry point override the choice.
+  const bool can_direct = bro::rqd::supports(M, K, layout, gemm_scale_kblocks(K));
+  bool direct = can_direct && (B == 32 || M * K <= ((int64_t)1 << 23));
+  if (flags & BRO_FLAG_RQ_TMA_RING) direct = false;
+  else if (flags & BRO_FLAG_RQ_DIRECT) direct = can_direct;
   if (direct)
     return bro::rqd::launch(x, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs, codes, scales, layout,
                             gemm_scale_kblocks(K), di.sm_count, st);
@@ -177,17 +192,12 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   const int64_t tiles = p.tiles_m * p.tiles_k;
   const int grid = (int)(tiles < di.sm_count ? tiles : di.sm_count);
 
-  // (All three instantiations share one function-pointer type, so the opt-in to large dynamic
-  // shared memory is keyed by the kernel's address, per device.)
+  // (All six instantiations share one function-pointer type, so the opt-in to large dynamic
+  // shared memory is kept per instantiation, per device.)
   auto go = [&](void (*kernel)(CUtensorMap, Params), int which) -> bro_status {
-    static bool attr_done[64][6] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!attr_done[dev][which]) {
-      bro_status r = set_smem(kernel, bro::rq::kSmemBytes);
-      if (r != BRO_OK) return r;
-      attr_done[dev][which] = true;
-    }
+    static bro::DeviceOnce once[6];
+    bro_status r = bro::device_once(once[which], nullptr, [&](int*) { return set_smem(kernel, bro::rq::kSmemBytes); });
+    if (r != BRO_OK) return r;
     return bro::cuda_ok(bro::launch_kernel(kernel, (unsigned)grid, bro::rq::kThreads, bro::rq::kSmemBytes, st, 1, tmx, p),
                         "rotate_quantize launch")
                ? BRO_OK
@@ -260,26 +270,48 @@ size_t bro_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
          align_up(bro_gemm_workspace_bytes(M, N, K), 1024);
 }
 
-bro_status bro_last_device_status(void* stream) {
+bro_status bro_last_device_status_ex(void* stream, int* site) {
+  if (site) *site = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaStreamSynchronize(st) != cudaSuccess) return BRO_ERR_CUDA;
+  if (!bro::cuda_ok(cudaStreamSynchronize(st), "cudaStreamSynchronize")) return BRO_ERR_CUDA;
   unsigned int v = 0, zero = 0;
-  if (cudaMemcpyFromSymbol(&v, bro::g_device_status, sizeof(v)) != cudaSuccess) return BRO_ERR_CUDA;
-  if (v != 0 && cudaMemcpyToSymbol(bro::g_device_status, &zero, sizeof(zero)) != cudaSuccess)
+  if (!bro::cuda_ok(cudaMemcpyFromSymbol(&v, bro::g_device_status, sizeof(v)), "read of the device status word"))
     return BRO_ERR_CUDA;
+  if (v != 0 && !bro::cuda_ok(cudaMemcpyToSymbol(bro::g_device_status, &zero, sizeof(zero)), "reset of the device status word"))
+    return BRO_ERR_CUDA;
+  if (site) *site = (int)(v >> 8);
   return (bro_status)(v & 0xFF);
+}
+
+bro_status bro_last_device_status(void* stream) { return bro_last_device_status_ex(stream, nullptr); }
+
+bro_status bro_selftest_expire_wait(uint64_t budget_ns, void* stream) {
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  if (budget_ns < 1000ull) budget_ns = 1000ull;
+  if (budget_ns > 100ull * 1000ull * 1000ull) budget_ns = 100ull * 1000ull * 1000ull;
+  expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(budget_ns);
+  return bro::cuda_ok(cudaGetLastError(), "self-test launch") ? BRO_OK : BRO_ERR_CUDA;
 }
 
 bro_status bro_rotate_quantize_mxfp4(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                      void* codes, void* scales, bro_layout layout, void* stream) {
-  return launch_rotate_quantize(x_bf16, M, K, ldx, block, nullptr, codes, scales, layout,
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, nullptr, codes, scales, layout, 0u,
+                                static_cast<cudaStream_t>(stream));
+}
+
+bro_status bro_rotate_quantize_mxfp4_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                        const void* signs_bf16, void* codes, void* scales, bro_layout layout,
+                                        uint32_t flags, void* stream) {
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, signs_bf16, codes, scales, layout, flags,
                                 static_cast<cudaStream_t>(stream));
 }
 
 bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                         const void* signs_bf16, void* codes, void* scales, bro_layout layout,
                                         void* stream) {
-  return launch_rotate_quantize(x_bf16, M, K, ldx, block, signs_bf16, codes, scales, layout,
+  return launch_rotate_quantize(x_bf16, M, K, ldx, block, signs_bf16, codes, scales, layout, 0u,
                                 static_cast<cudaStream_t>(stream));
 }
 
@@ -312,19 +344,19 @@ bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64
 
 bro_status bro_pack_weights_rs(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
                                const void* signs_bf16, void* wcodes, void* wscales, void* stream) {
-  return launch_rotate_quantize(w_bf16, N, K, ldw, block, signs_bf16, wcodes, wscales, BRO_LAYOUT_GEMM,
+  return launch_rotate_quantize(w_bf16, N, K, ldw, block, signs_bf16, wcodes, wscales, BRO_LAYOUT_GEMM, 0u,
                                 static_cast<cudaStream_t>(stream));
 }
 
 bro_status bro_pack_weights(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
                             void* wcodes, void* wscales, void* stream) {
-  return launch_rotate_quantize(w_bf16, N, K, ldw, block, nullptr, wcodes, wscales, BRO_LAYOUT_GEMM,
+  return launch_rotate_quantize(w_bf16, N, K, ldw, block, nullptr, wcodes, wscales, BRO_LAYOUT_GEMM, 0u,
                                 static_cast<cudaStream_t>(stream));
 }
 
 static bro_status gemm_impl(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
                             int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, bro_out_dtype out_dtype,
-                            void* workspace, size_t workspace_bytes, void* stream, bool w_static) {
+                            void* workspace, size_t workspace_bytes, uint32_t flags, void* stream, bool w_static) {
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0 || ldy < N) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (out_dtype != BRO_OUT_BF16 && out_dtype != BRO_OUT_F32) return BRO_ERR_SHAPE;
@@ -340,15 +372,13 @@ static bro_status gemm_impl(const void* acodes, const void* ascales, const void*
   DeviceInfo di;
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
-  // Default: one CTA per 128 x BN tile.  BRO_GEMM_PAIR=1 selects the two-CTA kernel (256 x 256
+  // Default: one CTA per 128 x BN tile.  BRO_FLAG_GEMM_PAIR selects the two-CTA kernel (256 x 256
   // tiles, cta_group::2), which moves a third fewer bytes from L2 but measured no faster.
-  bool pair = false;
-  if (const char* e = getenv("BRO_GEMM_PAIR")) pair = atoi(e) != 0;
-  if (pair)
+  if (flags & BRO_FLAG_GEMM_PAIR)
     return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, di.sm_count,
                               static_cast<cudaStream_t>(stream));
   return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,
-                           workspace_bytes, di.sm_count, static_cast<cudaStream_t>(stream), w_static);
+                           workspace_bytes, flags, di.sm_count, static_cast<cudaStream_t>(stream), w_static);
 }
 
 bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* wcodes,
@@ -356,13 +386,20 @@ bro_status bro_gemm_mxfp4(const void* acodes, const void* ascales, const void* w
                           bro_out_dtype out_dtype, void* workspace, size_t workspace_bytes,
                           void* stream) {
   // the weights may have been written by the kernel just before this one: no early fetch
-  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, out_dtype, workspace, workspace_bytes, stream,
-                   false);
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, out_dtype, workspace, workspace_bytes, 0u,
+                   stream, false);
+}
+
+bro_status bro_gemm_mxfp4_ex(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
+                             int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, bro_out_dtype out_dtype,
+                             void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, out_dtype, workspace, workspace_bytes, flags,
+                   stream, false);
 }
 
 static bro_status linear_impl(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs,
                               const void* wcodes, const void* wscales, int64_t N, void* y_bf16, int64_t ldy,
-                              void* workspace, size_t workspace_bytes, void* stream) {
+                              void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
   if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
   if (M == 0 || N == 0) return BRO_OK;
   if (!x_bf16 || !wcodes || !wscales || !y_bf16 || !workspace) return BRO_ERR_NULL;
@@ -372,20 +409,27 @@ static bro_status linear_impl(const void* x_bf16, int64_t M, int64_t K, int64_t 
   uint8_t* acodes = ws;
   uint8_t* ascales = acodes + align_up(bro_codes_bytes(M, K), 1024);
   uint8_t* gws = ascales + align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 1024);
-  bro_status rc = launch_rotate_quantize(x_bf16, M, K, ldx, block, signs, acodes, ascales, BRO_LAYOUT_GEMM,
+  bro_status rc = launch_rotate_quantize(x_bf16, M, K, ldx, block, signs, acodes, ascales, BRO_LAYOUT_GEMM, flags,
                                          static_cast<cudaStream_t>(stream));
   if (rc != BRO_OK) return rc;
   // The packed weights are older than the rotate+quantize kernel just enqueued, which signals its
   // dependents only after its own wait: the GEMM may fetch its first weight tiles early.
   return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
-                   bro_gemm_workspace_bytes(M, N, K), stream, true);
+                   bro_gemm_workspace_bytes(M, N, K), flags, stream, true);
 }
 
 bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* wcodes,
                       const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
                       size_t workspace_bytes, void* stream) {
   return linear_impl(x_bf16, M, K, ldx, block, nullptr, wcodes, wscales, N, y_bf16, ldy, workspace,
-                     workspace_bytes, stream);
+                     workspace_bytes, 0u, stream);
+}
+
+bro_status bro_linear_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs_bf16,
+                         const void* wcodes, const void* wscales, int64_t N, void* y_bf16, int64_t ldy,
+                         void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  return linear_impl(x_bf16, M, K, ldx, block, signs_bf16, wcodes, wscales, N, y_bf16, ldy, workspace,
+                     workspace_bytes, flags, stream);
 }
 
 bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs_bf16,
@@ -393,7 +437,7 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
                          void* workspace, size_t workspace_bytes, void* stream) {
   if (!signs_bf16) return BRO_ERR_NULL;
   return linear_impl(x_bf16, M, K, ldx, block, signs_bf16, wcodes, wscales, N, y_bf16, ldy, workspace,
-                     workspace_bytes, stream);
+                     workspace_bytes, 0u, stream);
 }
 
 bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block, const void* wcodes,
@@ -462,7 +506,7 @@ bro_status bro_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t l
   // (as in bro_linear: the packed weights are older than the kernel just enqueued, so the GEMM may
   // fetch its first weight tiles before that kernel has finished)
   return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gemm_sz ? gws : nullptr,
-                   gemm_sz, stream, true);
+                   gemm_sz, 0u, stream, true);
 }
 
 }  // extern "C"

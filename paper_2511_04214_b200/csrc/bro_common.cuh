@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <mutex>
+
 #include "../../include/bro.h"
 
 namespace bro {
@@ -17,6 +19,29 @@ inline bool cuda_ok(cudaError_t e, const char* what) {
   if (e == cudaSuccess) return true;
   snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s: %s", what, cudaGetErrorString(e));
   return false;
+}
+
+// One-time, per-device set-up of a kernel (shared-memory opt-in, occupancy query): host threads may
+// race to the first launch, so the "done" table is guarded.  `init` returns BRO_OK and a positive
+// value to remember; later calls on the same device get that value back without running it again.
+struct DeviceOnce {
+  std::mutex mu;
+  int value[64] = {};
+};
+template <typename Init>
+inline bro_status device_once(DeviceOnce& once, int* value_out, Init&& init) {
+  int dev = 0;
+  if (!cuda_ok(cudaGetDevice(&dev), "cudaGetDevice")) return BRO_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return BRO_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(once.mu);
+  if (once.value[dev] == 0) {
+    int v = 1;
+    const bro_status rc = init(&v);
+    if (rc != BRO_OK) return rc;
+    once.value[dev] = v > 0 ? v : 1;
+  }
+  if (value_out) *value_out = once.value[dev];
+  return BRO_OK;
 }
 
 // Launch with programmatic dependent launch enabled (and, if cluster_x > 1, that cluster width).
@@ -49,14 +74,15 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), unsigned grid, unsign
 // 0 = OK; otherwise (BRO_ERR_TIMEOUT) | (site << 8).  Kernels only ever move it away from 0.
 __device__ unsigned int g_device_status = 0u;
 
-// Upper bound on mbarrier polling before a wait is declared lost.  Each failed try_wait already
-// blocks for a hardware-defined interval, so this is on the order of a second.
-constexpr uint32_t kSpinLimit = 4u * 1000u * 1000u;
+// Time budget of one mbarrier wait, measured on the device's nanosecond timer (%globaltimer): a wait
+// that has not completed after this long is declared lost.  No wait of a healthy run lasts longer than
+// a kernel does (milliseconds); two seconds is far beyond that and still returns the GPU promptly.
+constexpr uint64_t kWaitBudgetNs = 2000ull * 1000ull * 1000ull;
 
 enum WaitSite : unsigned {
   SITE_RQ_FULL = 1, SITE_RQ_EMPTY = 2, SITE_RQ_DRAIN = 3,
   SITE_GEMM_FULL = 4, SITE_GEMM_EMPTY = 5, SITE_GEMM_ACC_FULL = 6, SITE_GEMM_ACC_EMPTY = 7,
-  SITE_GEMM_DRAIN = 8, SITE_GEMM_TMEM = 9
+  SITE_GEMM_DRAIN = 8, SITE_GEMM_TMEM = 9, SITE_SELF_TEST = 10
 };
 
 __device__ __forceinline__ void report_timeout(unsigned site) {
@@ -94,10 +120,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (after recording the site) if the phase never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned site) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false (after recording the site) if the phase has not completed within
+// `budget_ns`.  The first probe costs nothing extra; the timer is read once per 32 failed probes
+// (each failed try_wait already suspends the thread for a hardware-defined interval).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned site,
+                                          uint64_t budget_ns = kWaitBudgetNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  do {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+  } while (global_timer_ns() - t0 <= budget_ns);
   report_timeout(site);
   return false;
 }

@@ -26,8 +26,6 @@
 // common exit, where outstanding copies are awaited and TMEM is released.
 #pragma once
 
-#include <stdlib.h>
-
 #include "bro_common.cuh"
 
 namespace bro {
@@ -618,7 +616,7 @@ bro_status make_out_map(CUtensorMap* map, const void* y, int64_t M, int64_t N, i
 
 template <int BN>
 bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUtensorMap& tmw_half,
-                       const CUtensorMap& tmy, Params& p, int out_dtype, int sm_count, cudaStream_t st) {
+                       const CUtensorMap& tmy, Params& p, int out_dtype, uint32_t flags, int sm_count, cudaStream_t st) {
   using C = Cfg<BN>;
   p.tiles_m = (int)((p.M + kBM - 1) / kBM);
   p.tiles_n = (int)((p.N + BN - 1) / BN);
@@ -631,24 +629,22 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
   // weight bytes from HBM.
   p.raster_rows = (double)p.N * (double)p.K * (17.0 / 32.0) > 64.0 * 1024 * 1024 ? 12 : kRasterRows;
   // Rounds of the persistent grid: when the last round would leave at least half of the SMs idle,
-  // its tiles are cut into two half-width units each (BRO_GEMM_SPLIT=0 switches this off).
+  // its tiles are cut into two half-width units each (BRO_FLAG_GEMM_NO_SPLIT switches this off).
   int64_t grid = total < sm_count ? total : sm_count;
   const int64_t rem = total % sm_count;
-  bool split = BN == 256 && rem > 0 && 2 * rem <= sm_count;
-  if (const char* e = getenv("BRO_GEMM_SPLIT")) split = split && atoi(e) != 0;
+  const bool split = BN == 256 && rem > 0 && 2 * rem <= sm_count && !(flags & BRO_FLAG_GEMM_NO_SPLIT);
   p.full_units = (int)(split ? total - rem : total);
   p.total_units = (int)(split ? total + rem : total);
   if (split && p.total_units < sm_count) grid = p.total_units;
   auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, Params), int which) -> bro_status {
-    static bool attr_done[64][2] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!attr_done[dev][which]) {
-      if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes),
-                   "cudaFuncSetAttribute(gemm)"))
-        return BRO_ERR_CUDA;
-      attr_done[dev][which] = true;
-    }
+    static DeviceOnce once[2];      // (per BN through the template, per output type through `which`)
+    const bro_status rc = device_once(once[which], nullptr, [&](int*) {
+      return cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes),
+                     "cudaFuncSetAttribute(gemm)")
+                 ? BRO_OK
+                 : BRO_ERR_CUDA;
+    });
+    if (rc != BRO_OK) return rc;
     return cuda_ok(launch_kernel(kernel, (unsigned)grid, kThreads, C::kSmemBytes, st, 1, tma, tmw, tmw_half, tmy, p),
                    "gemm_mxfp4 launch")
                ? BRO_OK
@@ -662,10 +658,10 @@ bro_status launch_tile(const CUtensorMap& tma, const CUtensorMap& tmw, const CUt
 // the library's own rotate+quantize and signals its dependents only after its own wait).
 inline bro_status launch(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
                          int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, void* /*ws*/,
-                         size_t /*ws_bytes*/, int sm_count, cudaStream_t st, bool w_static = false) {
-  int bn = 256;
-  if (const char* e = getenv("BRO_GEMM_TILE_N")) bn = atoi(e) == 128 ? 128 : 256;
-  else if (N <= 128) bn = 128;
+                         size_t /*ws_bytes*/, uint32_t flags, int sm_count, cudaStream_t st, bool w_static = false) {
+  int bn = N <= 128 ? 128 : 256;
+  if (flags & BRO_FLAG_GEMM_TILE_N128) bn = 128;
+  else if (flags & BRO_FLAG_GEMM_TILE_N256) bn = 256;
   Params p;
   p.ascales = static_cast<const uint8_t*>(ascales);
   p.wscales = static_cast<const uint8_t*>(wscales);
@@ -694,8 +690,8 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   CUtensorMap tmw_half;       // the same weights seen through a box of half as many rows
   rc = make_codes_map(&tmw_half, wcodes, N, K, bn / 2);
   if (rc != BRO_OK) return rc;
-  return bn == 256 ? launch_tile<256>(tma, tmw, tmw_half, tmy, p, out_dtype, sm_count, st)
-                   : launch_tile<128>(tma, tmw, tmw_half, tmy, p, out_dtype, sm_count, st);
+  return bn == 256 ? launch_tile<256>(tma, tmw, tmw_half, tmy, p, out_dtype, flags, sm_count, st)
+                   : launch_tile<128>(tma, tmw, tmw_half, tmy, p, out_dtype, flags, sm_count, st);
 }
 
 }  // namespace gemm

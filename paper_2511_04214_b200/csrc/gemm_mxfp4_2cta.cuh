@@ -290,21 +290,21 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   }
   auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, Params),
                 int which) -> bro_status {
-    static int pairs_of[64][2] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (pairs_of[dev][which] == 0) {
+    static DeviceOnce once[2];
+    int resident = 0;
+    const bro_status rc = device_once(once[which], &resident, [&](int* n) {
       if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
                    "cudaFuncSetAttribute(gemm pair)"))
         return BRO_ERR_CUDA;
-      const int n = max_resident_pairs(kernel, sm_count);
-      if (n <= 0) {
+      *n = max_resident_pairs(kernel, sm_count);
+      if (*n <= 0) {
         snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "no resident 2-CTA cluster fits on this device");
         return BRO_ERR_CUDA;
       }
-      pairs_of[dev][which] = n;
-    }
-    const int64_t pairs = total < pairs_of[dev][which] ? total : pairs_of[dev][which];
+      return BRO_OK;
+    });
+    if (rc != BRO_OK) return rc;
+    const int64_t pairs = total < resident ? total : resident;
     return cuda_ok(launch_kernel(kernel, (unsigned)(2 * pairs), kThreads, kSmemBytes, st, 2, tma, tmw, tmsfa, tmsfb,
                                  tmy, p),
                    "gemm_mxfp4 pair launch")

@@ -142,17 +142,16 @@ inline bool supports(int64_t M, int64_t K, bro_layout layout, int64_t scale_kblo
 template <int LOG2B, bool SIGNS, bool STATS>
 inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
   auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS, STATS>;
-  static int blocks_per_sm[64] = {};
-  int dev = 0;
-  cudaGetDevice(&dev);
-  if (blocks_per_sm[dev] == 0) {
-    int n = 0;
-    if (!cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0), "occupancy(rotate_quantize_direct)"))
-      return BRO_ERR_CUDA;
-    blocks_per_sm[dev] = n > 0 ? n : 1;
-  }
+  static DeviceOnce once;            // (one per template instantiation)
+  int blocks_per_sm = 1;
+  const bro_status rc = device_once(once, &blocks_per_sm, [&](int* n) {
+    return cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, kernel, kThreads, 0), "occupancy(rotate_quantize_direct)")
+               ? BRO_OK
+               : BRO_ERR_CUDA;
+  });
+  if (rc != BRO_OK) return rc;
   const int64_t want = ((int64_t)p.total_tasks + kWarps - 1) / kWarps;
-  const int64_t cap = (int64_t)sm_count * blocks_per_sm[dev];
+  const int64_t cap = (int64_t)sm_count * blocks_per_sm;
   const unsigned grid = (unsigned)(want < cap ? want : cap);
   return cuda_ok(launch_kernel(kernel, grid, kThreads, 0, st, 1, p), "rotate_quantize_direct launch") ? BRO_OK
                                                                                                        : BRO_ERR_CUDA;

@@ -43,11 +43,11 @@ def sample_points(M, N, rng, n_random):
     return np.concatenate(pm).astype(np.int64), np.concatenate(pn).astype(np.int64)
 
 
-def check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, block, n_random, seed):
+def check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, block, n_random, seed, flags=0):
     M, K = x.shape
     ws = bro.alloc_workspace(bro.linear_workspace_bytes(M, N, K))
     y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-    bro.linear(x.cuda(), block, wcodes, wscales, N, y, ws)
+    bro.linear(x.cuda(), block, wcodes, wscales, N, y, ws, flags=flags)
     assert bro.last_device_status() == 0
     ac_ref, as_ref = oracle.rotate_quantize_mxfp4(synth.bf16_bits(x), block)
     nc = bro.codes_bytes(M, K)
@@ -91,6 +91,22 @@ def test_llm_shaped_layers_full_size(bro, name, index):
     check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, 32, 100000, seed)
 
 
+@pytest.mark.parametrize("variant", ["pair", "tile_n128", "no_split"])
+def test_other_gemm_kernels_on_a_many_tile_shape(bro, variant):
+    """M = 4096, K = 4096, N = 14336 (1792 tiles of 128 x 256: twelve per CTA, across raster bands)
+    through the GEMM variants the library does not pick by itself — the two-CTA kernel, 128-column
+    tiles, and the schedule without half-width units — so that their accumulator ping-pong over many
+    tiles per CTA is compared with the oracle too."""
+    cfg = synth.CONFIGS["cfg3"]
+    M, K, N = cfg["shapes"][1]
+    seed = synth.config_seed("cfg3", 1)
+    x = synth.activations(M, K, seed=seed, recipe=cfg["recipe"])
+    w = synth.weights(N, K, seed=seed)
+    wc_ref, ws_ref, wcodes, wscales = pack_both(bro, w, 32)
+    flags = {"pair": bro.FLAG_GEMM_PAIR, "tile_n128": bro.FLAG_GEMM_TILE_N128, "no_split": bro.FLAG_GEMM_NO_SPLIT}[variant]
+    check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, 32, 100000, seed, flags=flags)
+
+
 @pytest.fixture(scope="module")
 def packed_70b(bro):
     cfg = synth.CONFIGS["cfg5"]
@@ -124,3 +140,22 @@ def test_block_sweep_tensor_full_size(bro):
         rc, rs = oracle.rotate_quantize_mxfp4(bits, block)
         assert np.array_equal(codes.cpu().numpy(), rc), f"codes differ, block {block}"
         assert np.array_equal(to_canonical(scales.cpu().numpy(), M, K), rs), f"scales differ, block {block}"
+
+
+@pytest.mark.parametrize("block", [32, 64, 128])
+@pytest.mark.parametrize("form", ["default", "direct", "tma_ring"])
+def test_block_sweep_tensor_randomised_rotation_both_kernels(bro, block, form):
+    """The same [16384, 4096] tensor with the randomised rotation diag(s) H / sqrt(block) (Sec. 5.1),
+    whole tensor, through the library's own choice at this size and through each block kernel forced."""
+    cfg = synth.CONFIGS["cfg4"]
+    M, K, _ = cfg["shapes"][0]
+    x = synth.activations(M, K, seed=cfg["seed"], recipe=cfg["recipe"])
+    signs = synth.rotation_signs(K, seed=cfg["seed"])
+    flags = {"default": 0, "direct": bro.FLAG_RQ_DIRECT, "tma_ring": bro.FLAG_RQ_TMA_RING}[form]
+    codes = bro.alloc_codes(M, K)
+    scales = bro.alloc_scales(M, K, bro.LAYOUT_GEMM)
+    bro.rotate_quantize_mxfp4(x.cuda(), block, codes, scales, bro.LAYOUT_GEMM, flags=flags, signs=signs.cuda())
+    assert bro.last_device_status() == 0
+    rc, rs = oracle.rotate_quantize_mxfp4(synth.bf16_bits(x), block, synth.bf16_bits(signs))
+    assert np.array_equal(codes.cpu().numpy(), rc), f"codes differ, block {block}"
+    assert np.array_equal(to_canonical(scales.cpu().numpy(), M, K), rs), f"scales differ, block {block}"

@@ -2,8 +2,6 @@
 CPU oracle's fp64 sums.  Tolerance (fp32 result): |y - y_ref| <= 1e-5 * sum_k |a_k w_k| + 1e-6.
 bf16 output: within that tolerance plus half a bf16 ulp of y_ref, and bit-identical to the
 round-to-nearest-even bf16 of the same kernel's fp32 result."""
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -28,7 +26,7 @@ def upload_operand(codes: np.ndarray, scales_canon: np.ndarray):
     return c, s
 
 
-def gpu_gemm(bro, ac, asc, wc, wsc, dtype, ldy=None):
+def gpu_gemm(bro, ac, asc, wc, wsc, dtype, ldy=None, flags=0):
     M, K = ac.shape[0], ac.shape[1] * 2
     N = wc.shape[0]
     a_c, a_s = upload_operand(ac, asc)
@@ -37,7 +35,8 @@ def gpu_gemm(bro, ac, asc, wc, wsc, dtype, ldy=None):
     esz = 2 if dtype == torch.bfloat16 else 4
     buf = Guarded(M * ldy * esz, fill=0x7F)
     y = buf.view.view(dtype).view(M, ldy)[:, :N]
-    bro.gemm_mxfp4(a_c, a_s, w_c, w_s, M, N, K, y)
+    ws = bro.alloc_workspace(bro.gemm_workspace_bytes(M, N, K))
+    bro.gemm_mxfp4(a_c, a_s, w_c, w_s, M, N, K, y, workspace=ws, flags=flags)
     assert bro.last_device_status() == 0
     buf.check()
     if ldy > N:   # the gap between rows must be untouched
@@ -60,11 +59,11 @@ def check_bf16(y16, y32_dev, y_ref, S):
     return expect
 
 
-def run_case(bro, ac, asc, wc, wsc, ldy=None):
+def run_case(bro, ac, asc, wc, wsc, ldy=None, flags=0):
     y_ref, S = oracle.gemm_mxfp4(ac, asc, wc, wsc)
-    y32, y32_dev = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32, ldy)
+    y32, y32_dev = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32, ldy, flags)
     check_f32(y32, y_ref, S)
-    y16, y16_dev = gpu_gemm(bro, ac, asc, wc, wsc, torch.bfloat16, ldy)
+    y16, y16_dev = gpu_gemm(bro, ac, asc, wc, wsc, torch.bfloat16, ldy, flags)
     expect = check_bf16(y16, y32_dev, y_ref, S)
     assert torch.equal(y16_dev.contiguous().view(torch.int16), expect.contiguous().view(torch.int16))
 
@@ -77,22 +76,13 @@ def quantized_pair(M, N, K, seed, block=32, recipe=synth.HEAVY_RECIPE):
     return x, w, ac, asc, wc, wsc
 
 
-@pytest.fixture(params=["cta1_n128", "cta1_n256", "pair"])
-def tile_n(request):
-    """Force each GEMM kernel variant in turn: the single-CTA kernel with 128- or 256-column tiles,
-    and the two-CTA (cta_group::2) kernel with 256 x 256 tiles."""
-    saved = {k: os.environ.get(k) for k in ("BRO_GEMM_TILE_N", "BRO_GEMM_PAIR")}
-    if request.param == "pair":
-        os.environ["BRO_GEMM_PAIR"] = "1"
-    else:
-        os.environ["BRO_GEMM_PAIR"] = "0"
-        os.environ["BRO_GEMM_TILE_N"] = request.param[-3:]
-    yield request.param
-    for k, v in saved.items():
-        if v is None:
-            os.environ.pop(k, None)
-        else:
-            os.environ[k] = v
+@pytest.fixture(params=["default", "cta1_n128", "cta1_n256", "pair"])
+def tile_n(request, bro):
+    """Each GEMM kernel variant in turn, as the `flags` word of bro_gemm_mxfp4_ex: the library's own
+    choice, the single-CTA kernel forced to 128- or 256-column tiles, and the two-CTA (cta_group::2)
+    kernel with 256 x 256 tiles."""
+    return {"default": 0, "cta1_n128": bro.FLAG_GEMM_TILE_N128, "cta1_n256": bro.FLAG_GEMM_TILE_N256,
+            "pair": bro.FLAG_GEMM_PAIR}[request.param]
 
 
 def test_unit_scales_small_integers_exact(bro, tile_n):
@@ -105,7 +95,7 @@ def test_unit_scales_small_integers_exact(bro, tile_n):
     asc = np.full((M, K // 32), 127, dtype=np.uint8)
     wsc = np.full((N, K // 32), 127, dtype=np.uint8)
     y_ref, S = oracle.gemm_mxfp4(ac, asc, wc, wsc)
-    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32)
+    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32, flags=tile_n)
     assert np.array_equal(y32, y_ref)
 
 
@@ -123,20 +113,20 @@ def test_scale_bytes_reach_the_right_rows_and_groups(bro, tile_n):
     asc = rng.integers(110, 140, size=(M, K // 32), dtype=np.uint8)
     wsc = rng.integers(110, 140, size=(N, K // 32), dtype=np.uint8)
     y_ref, S = oracle.gemm_mxfp4(ac, asc, wc, wsc)
-    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32)
+    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32, flags=tile_n)
     assert np.array_equal(y32, y_ref)
 
 
 def test_config1_full_output(bro, tile_n):
     _, _, ac, asc, wc, wsc = quantized_pair(64, 2048, 2048, seed=0, recipe=synth.CFG1_RECIPE)
-    run_case(bro, ac, asc, wc, wsc)
+    run_case(bro, ac, asc, wc, wsc, flags=tile_n)
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (129, 136, 160), (300, 520, 416), (128, 256, 288),
                                    (257, 129, 1024), (64, 384, 3072), (700, 1300, 512), (2304, 1000, 768)])
 def test_ragged_shapes(bro, tile_n, M, N, K):
     _, _, ac, asc, wc, wsc = quantized_pair(M, N, K, seed=M + N + K)
-    run_case(bro, ac, asc, wc, wsc)
+    run_case(bro, ac, asc, wc, wsc, flags=tile_n)
 
 
 @pytest.mark.parametrize("M,N,K", [(128 * 19, 2048, 256), (128 * 5, 300, 512), (128 * 3, 4 * 256 + 40, 288)])
@@ -146,16 +136,12 @@ def test_half_width_units_of_the_last_round(bro, M, N, K):
     half-width units each.  Includes a ragged N whose last half-width unit lies beyond N."""
     _, _, ac, asc, wc, wsc = quantized_pair(M, N, K, seed=M + N)
     run_case(bro, ac, asc, wc, wsc)
-    os.environ["BRO_GEMM_SPLIT"] = "0"
-    try:
-        run_case(bro, ac, asc, wc, wsc)
-    finally:
-        del os.environ["BRO_GEMM_SPLIT"]
+    run_case(bro, ac, asc, wc, wsc, flags=bro.FLAG_GEMM_NO_SPLIT)
 
 
 def test_row_stride_of_y(bro, tile_n):
     _, _, ac, asc, wc, wsc = quantized_pair(130, 136, 256, seed=9)
-    run_case(bro, ac, asc, wc, wsc, ldy=136 + 24)
+    run_case(bro, ac, asc, wc, wsc, ldy=136 + 24, flags=tile_n)
 
 
 def test_wide_scale_range_and_all_positive_stress(bro, tile_n):
@@ -168,7 +154,7 @@ def test_wide_scale_range_and_all_positive_stress(bro, tile_n):
     asc = rng.integers(87, 167, size=(M, K // 32), dtype=np.uint8)
     wsc = rng.integers(87, 167, size=(N, K // 32), dtype=np.uint8)
     y_ref, S = oracle.gemm_mxfp4(ac, asc, wc, wsc)
-    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32)
+    y32, _ = gpu_gemm(bro, ac, asc, wc, wsc, torch.float32, flags=tile_n)
     # with an 80-binade spread the absolute floor 1e-6 is meaningless: relative criterion only
     assert np.all(np.abs(y32 - y_ref) <= 1e-5 * S)
     K = 14336
@@ -176,7 +162,7 @@ def test_wide_scale_range_and_all_positive_stress(bro, tile_n):
     wc = (rng.integers(0, 256, size=(128, K // 2), dtype=np.uint8) & 0x77)
     asc = rng.integers(125, 130, size=(64, K // 32), dtype=np.uint8)
     wsc = rng.integers(125, 130, size=(128, K // 32), dtype=np.uint8)
-    run_case(bro, ac, asc, wc, wsc)
+    run_case(bro, ac, asc, wc, wsc, flags=tile_n)
 
 
 def test_linear_end_to_end_config1(bro):

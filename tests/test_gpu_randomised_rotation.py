@@ -18,12 +18,21 @@ def bro():
     return binding
 
 
-def compare(bro, x, signs, block, layout):
+@pytest.fixture(params=["default", "direct", "tma_ring"])
+def form(request, bro):
+    """The library's own kernel choice, then each of the two block kernels forced (flags of the _ex entry point)."""
+    return {"default": 0, "direct": bro.FLAG_RQ_DIRECT, "tma_ring": bro.FLAG_RQ_TMA_RING}[request.param]
+
+
+def compare(bro, x, signs, block, layout, flags=0):
     M, K = x.shape
     rc, rs = oracle.rotate_quantize_mxfp4(synth.bf16_bits(x), block, synth.bf16_bits(signs))
     codes = Guarded(bro.codes_bytes(M, K))
     scales = Guarded(bro.scales_bytes(M, K, layout))
-    bro.rotate_quantize_mxfp4_rs(x.cuda(), block, signs.cuda(), codes.view, scales.view, layout)
+    if flags:
+        bro.rotate_quantize_mxfp4(x.cuda(), block, codes.view, scales.view, layout, flags=flags, signs=signs.cuda())
+    else:
+        bro.rotate_quantize_mxfp4_rs(x.cuda(), block, signs.cuda(), codes.view, scales.view, layout)
     assert bro.last_device_status() == 0
     codes.check(); scales.check()
     gs = scales.numpy()
@@ -33,12 +42,16 @@ def compare(bro, x, signs, block, layout):
 
 
 @pytest.mark.parametrize("block", [32, 64, 128, 0])
-@pytest.mark.parametrize("M,K", [(64, 2048), (300, 1024), (7, 256)])
-def test_codes_and_scales_bit_exact(bro, block, M, K):
+@pytest.mark.parametrize("M,K", [(64, 2048), (300, 1024), (7, 256), (513, 2176), (1024, 4096)])
+def test_codes_and_scales_bit_exact(bro, form, block, M, K):
+    if block and K % block:
+        pytest.skip("K not a multiple of the block")
+    if block == 0 and K & (K - 1):
+        pytest.skip("the full-dimension rotation needs a power-of-two K")
     x = synth.activations(M, K, seed=40 + M)
     signs = synth.rotation_signs(K, seed=K)
-    compare(bro, x, signs, block, 1)
-    compare(bro, x, signs, block, 0)
+    compare(bro, x, signs, block, 1, form)
+    compare(bro, x, signs, block, 0, form)
 
 
 def test_ragged_k_and_all_plus_signs(bro):

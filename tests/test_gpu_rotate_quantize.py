@@ -17,11 +17,19 @@ def bro():
     return binding
 
 
-def run_gpu(bro, x_dev, block, layout, ld=None):
+@pytest.fixture(params=["default", "direct", "tma_ring"])
+def form(request, bro):
+    """The two kernels behind block 32 / 64 / 128 — the register-streaming one and the shared-memory
+    ring fed by TMA — each forced through the `flags` word of bro_rotate_quantize_mxfp4_ex, next to the
+    library's own choice.  (The full-dimension rotation has one kernel; it ignores the flags.)"""
+    return {"default": 0, "direct": bro.FLAG_RQ_DIRECT, "tma_ring": bro.FLAG_RQ_TMA_RING}[request.param]
+
+
+def run_gpu(bro, x_dev, block, layout, flags=0):
     M, K = x_dev.shape
     codes = Guarded(bro.codes_bytes(M, K))
     scales = Guarded(bro.scales_bytes(M, K, layout))
-    bro.rotate_quantize_mxfp4(x_dev, block, codes.view, scales.view, layout)
+    bro.rotate_quantize_mxfp4(x_dev, block, codes.view, scales.view, layout, flags=flags)
     assert bro.last_device_status() == 0
     codes.check()
     scales.check()
@@ -39,10 +47,10 @@ def run_gpu(bro, x_dev, block, layout, ld=None):
     return c, s
 
 
-def compare(bro, x_cpu, block, layout):
+def compare(bro, x_cpu, block, layout, flags=0):
     bits = synth.bf16_bits(x_cpu)
     rc, rs = oracle.rotate_quantize_mxfp4(bits, block)
-    gc, gs = run_gpu(bro, x_cpu.cuda(), block, layout)
+    gc, gs = run_gpu(bro, x_cpu.cuda(), block, layout, flags)
     assert np.array_equal(gs, rs), f"scale mismatch: {(gs != rs).sum()} of {rs.size}"
     bad = gc != rc
     assert not bad.any(), f"code mismatch: {bad.sum()} bytes of {rc.size}, first at {np.argwhere(bad)[0]}"
@@ -50,19 +58,22 @@ def compare(bro, x_cpu, block, layout):
 
 @pytest.mark.parametrize("block", [32, 64, 128, 0])
 @pytest.mark.parametrize("layout", [0, 1])
-def test_config1_activations(bro, block, layout):
+def test_config1_activations(bro, form, block, layout):
     x = synth.activations(64, 2048, seed=0, recipe=synth.CFG1_RECIPE)
-    compare(bro, x, block, layout)
+    compare(bro, x, block, layout, form)
 
 
-@pytest.mark.parametrize("M,K", [(1, 32), (1, 128), (7, 160), (129, 416), (300, 1024), (513, 2176)])
-@pytest.mark.parametrize("block", [32, 64, 128])
-def test_ragged_shapes(bro, M, K, block):
-    if K % block:
-        pytest.skip("K not a multiple of the block")
+RAGGED = [(M, K, b) for (M, K) in [(1, 32), (1, 128), (7, 160), (129, 416), (300, 1024), (513, 2176), (1024, 4096)]
+          for b in (32, 64, 128) if K % b == 0]
+
+
+@pytest.mark.parametrize("M,K,block", RAGGED)
+def test_ragged_shapes(bro, form, M, K, block):
+    """Ragged in both directions (rows beyond M inside the last 128-row tile, K that ends inside a
+    128-column tile or a 256-column scale block) and several row tiles, through both kernels."""
     x = synth.activations(M, K, seed=100 + M + K)
-    compare(bro, x, block, 1)
-    compare(bro, x, block, 0)
+    compare(bro, x, block, 1, form)
+    compare(bro, x, block, 0, form)
 
 
 @pytest.mark.parametrize("K", [32, 64, 256, 1024, 2048, 4096, 8192, 16384, 32768])
@@ -88,18 +99,18 @@ def test_weights_path_and_heavy_tails(bro):
         compare(bro, x, block, 1)
 
 
-def test_row_stride_larger_than_K(bro):
+def test_row_stride_larger_than_K(bro, form):
     base = synth.activations(200, 512, seed=77)
     x_dev = base.cuda()[:, 64:64 + 256]                  # ldx = 512, K = 256, offset 128 bytes
     assert x_dev.stride(0) == 512
     sub = base[:, 64:64 + 256].contiguous()
     rc, rs = oracle.rotate_quantize_mxfp4(synth.bf16_bits(sub), 64)
-    gc, gs = run_gpu(bro, x_dev, 64, 0)
+    gc, gs = run_gpu(bro, x_dev, 64, 0, form)
     assert np.array_equal(gc, rc) and np.array_equal(gs, rs)
 
 
 @pytest.mark.parametrize("block", [32, 64, 128, 0])
-def test_degenerate_values(bro, block):
+def test_degenerate_values(bro, form, block):
     """All-zero rows, negative zeros, groups far below / above the fast-path exponent window,
     exact cancellations (equal neighbours) and bf16 subnormals."""
     K = 256
@@ -117,8 +128,8 @@ def test_degenerate_values(bro, block):
     x32 = torch.from_numpy(np.stack(rows))
     x = x32.to(torch.bfloat16)
     assert torch.isfinite(x.float()).all()
-    compare(bro, x, block, 0)
-    compare(bro, x, block, 1)
+    compare(bro, x, block, 0, form)
+    compare(bro, x, block, 1, form)
 
 
 def test_config4_slice_all_blocks(bro):

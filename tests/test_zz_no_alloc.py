@@ -13,6 +13,7 @@ This file sorts last on purpose: a run that stops at the first failure has then 
 through every other test."""
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
@@ -55,6 +56,15 @@ def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row(bro):
     assert bro.last_device_status() == 0
     for y, (_, _, _, _, _, expect) in zip(outs, prepared):
         assert torch.equal(y.view(torch.int16), expect.view(torch.int16))
+    # ... and the second problem directly against the CPU oracle, within the GEMM tolerance of the
+    # other tests (fp32 criterion plus half a bf16 ulp)
+    import oracle
+    (M, K, N, seed, block) = cases[1]
+    xb = synth.bf16_bits(synth.activations(M, K, seed=seed))
+    wc_ref, ws_ref = oracle.pack_weights(synth.bf16_bits(synth.weights(N, K, seed=seed)), block)
+    y_ref, S = oracle.linear(xb, block, wc_ref, ws_ref)
+    got = outs[1].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - y_ref) <= 1e-5 * S + 1e-6 + np.abs(y_ref) * 2.0 ** -8)
 
 
 def test_static_scratch_rejects_a_problem_that_does_not_fit(bro):
