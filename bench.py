@@ -3,15 +3,20 @@
 
 One *step* = one pass of the whole hot path — fused block-Hadamard rotation + MXFP4 quantisation
 of the activations, then the block-scaled MXFP4 GEMM against pre-packed weights — over every
-shape of the workload (default: the three LLaMA-3.2-1B-shaped layers, M = 2048 tokens).
+shape of the workload.  Default workload: cfg5, the 70B-shaped layer K = 8192, N = 28672 with
+M in {1, 16, 128, 1024, 8192, 32768} tokens (the largest single-GPU workload of the five).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg1|cfg2|cfg3|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `value` is device-timed throughput with inputs resident in HBM;
 `e2e` is the same metric through the host-buffer entry point (H2D of x and D2H of y inside the
-timed region); `roofline` describes the dominant kernel (the GEMM) timed per launch with CUDA
-events; `cpu_baseline` is the CPU oracle on a bounded sample.  With --gpus N > 1 (launched by
-torchrun) every rank runs an independent replica — the path has no cross-GPU exchange.
+timed region); `roofline` describes the dominant kernel (the GEMM on the tensor-bound shapes,
+M >= 1024) timed per launch with CUDA events, `decode` the weight-streaming shapes (M <= 128)
+against the HBM copy bandwidth; `per_config` repeats the per-kernel figures for the other
+workloads (cfg2, cfg3 and the block-size sweep cfg4) in the same process; `cpu_baseline` is the
+CPU oracle on a bounded sample.  With --gpus N > 1 every rank runs an independent replica — the
+path has no cross-GPU exchange; when no launcher has set WORLD_SIZE the script starts its N ranks
+itself.
 """
 from __future__ import annotations
 
@@ -31,6 +36,8 @@ METRIC = "MXFP4 W4A4 linear TFLOPS (rotate+quantize+GEMM)"
 UNIT = "TFLOP/s"
 L2_BYTES = 126 * 1024 * 1024
 FP4_OVER_BF16 = 4.0          # nominal dense fp4 : bf16 tensor throughput ratio on B200 (9 : 2.25)
+NOMINAL_FP4_TFLOPS = 9000.0  # dense FP4 tensor peak of one B200 (vendor figure)
+NOMINAL_HBM_GBS = 8000.0     # vendor HBM3e figure
 
 
 def workload_shapes(name):
@@ -131,7 +138,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -243,6 +250,227 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+class Layers:
+    """Device-resident inputs of one workload: per shape a ring of independent activation / weight /
+    output / workspace sets, so that consecutive launches never find their operands in L2 (126 MB)."""
+
+    def __init__(self, bro, synth, cfg, shapes, idx, block, dev, randomised=False, max_ring=8):
+        import torch
+        self.bro, self.shapes, self.block, self.dev = bro, shapes, block, dev
+        self.per_step_bytes = sum(M * K * 2 + N * K // 2 + M * N * 2 for (M, K, N) in shapes)
+        self.ring = max(2, min(max_ring, -(-3 * L2_BYTES // self.per_step_bytes)))
+        # --randomised: R_i = diag(s) H / sqrt(block) with a seeded +-1 vector per layer (Sec. 5.1)
+        self.signs = [synth.rotation_signs(K, seed=cfg["seed"] + idx[j]).to(dev) if randomised else None
+                      for j, (M, K, N) in enumerate(shapes)]
+        self.sets = []
+        wcache = {}
+        for j, (M, K, N) in enumerate(shapes):
+            i = idx[j]
+            wkey = (N, K, cfg["seed"] + i)
+            if wkey not in wcache:
+                wcache.clear()                  # (one bf16 weight matrix on the device at a time)
+                wcache[wkey] = synth.weights(N, K, seed=cfg["seed"] + i).to(dev)
+            w = wcache[wkey]
+            x0 = synth.activations(M, K, seed=cfg["seed"] + i, recipe=cfg["recipe"]).to(dev)
+            ws_bytes = bro.linear_workspace_bytes(M, N, K)
+            per_ring = []
+            for r in range(self.ring):
+                wcodes = bro.alloc_codes(N, K, dev)
+                wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM, dev)
+                if self.signs[j] is not None:
+                    bro.pack_weights_rs(w, block, self.signs[j], wcodes, wscales)   # offline, untimed
+                else:
+                    bro.pack_weights(w, block, wcodes, wscales)                     # offline, untimed
+                x = x0 if r == 0 else x0.roll(r * 7, 0).contiguous()   # same statistics, separate memory
+                per_ring.append({"x": x, "wcodes": wcodes, "wscales": wscales,
+                                 "y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+                                 "ws": bro.alloc_workspace(ws_bytes, dev)})
+            self.sets.append(per_ring)
+        wcache.clear()
+        torch.cuda.synchronize()
+
+    def step(self, r):
+        bro = self.bro
+        for i, (M, K, N) in enumerate(self.shapes):
+            s = self.sets[i][r % self.ring]
+            if self.signs[i] is not None:
+                bro.linear_rs(s["x"], self.block, self.signs[i], s["wcodes"], s["wscales"], N, s["y"], s["ws"])
+            else:
+                bro.linear(s["x"], self.block, s["wcodes"], s["wscales"], N, s["y"], s["ws"])
+
+    def views(self, i, r):
+        M, K, N = self.shapes[i]
+        s = self.sets[i][r]
+        nc = self.bro.codes_bytes(M, K)
+        off = (nc + 1023) // 1024 * 1024
+        sc = self.bro.scales_bytes(M, K, self.bro.LAYOUT_GEMM)
+        off2 = (off + sc + 1023) // 1024 * 1024
+        return s, s["ws"][:nc], s["ws"][off:off + sc], s["ws"][off2:]
+
+    def flops_per_step(self):
+        return sum(2.0 * M * K * N for (M, K, N) in self.shapes)
+
+
+def time_steps(layers, steps, warmup, use_graph, barrier, sampler=None):
+    """Device time of `steps` whole-layer steps (rounded up to a multiple of the ring when replaying a
+    CUDA graph of one ring of steps).  Returns (milliseconds on this rank, steps actually run)."""
+    import torch
+    for i in range(max(warmup, 3)):            # also sets kernel attributes before any graph capture
+        layers.step(i)
+    torch.cuda.synchronize()
+    graph = None
+    ring = layers.ring
+    if use_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for r in range(ring):
+                layers.step(r)
+        graph.replay()
+        torch.cuda.synchronize()
+        replays = max(1, -(-steps // ring))
+        steps = replays * ring
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler is not None:
+        sampler.mark("t0")
+    e0.record()
+    if graph is not None:
+        for _ in range(replays):
+            graph.replay()
+    else:
+        for i in range(steps):
+            layers.step(i)
+    e1.record()
+    barrier()
+    if sampler is not None:
+        sampler.mark("t1")
+    return e0.elapsed_time(e1), steps
+
+
+def time_kernels(layers, groups):
+    """Per-kernel device times: the two C-ABI calls bro_linear makes, each timed with CUDA events
+    around a group of `ring` back-to-back launches (one per ring set, so no launch finds its operands
+    in L2); per-launch time = group time / ring.  Timing every launch with its own pair of events adds
+    microseconds of event latency to kernels that only run for ten.  Returns (rq_ms, gemm_ms) per shape."""
+    import torch
+    bro, shapes, ring, block = layers.bro, layers.shapes, layers.ring, layers.block
+    rq_ev = [[] for _ in shapes]
+    gemm_ev = [[] for _ in shapes]
+    torch.cuda._sleep(int(4e7))        # hold the stream (~20 ms) while the launches below queue up
+    for it in range(groups + 2):
+        for i, (M, K, N) in enumerate(shapes):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            for r in range(ring):
+                s, acodes, ascales, _ = layers.views(i, r)
+                if layers.signs[i] is not None:
+                    bro.rotate_quantize_mxfp4_rs(s["x"], block, layers.signs[i], acodes, ascales, bro.LAYOUT_GEMM)
+                else:
+                    bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
+            ev[1].record()
+            for r in range(ring):
+                s, acodes, ascales, gws = layers.views(i, r)
+                bro.gemm_mxfp4(acodes, ascales, s["wcodes"], s["wscales"], M, N, K, s["y"], workspace=gws)
+            ev[2].record()
+            if it >= 2:
+                rq_ev[i].append((ev[0], ev[1]))
+                gemm_ev[i].append((ev[1], ev[2]))
+    torch.cuda.synchronize()
+    rq_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in rq_ev]
+    gemm_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in gemm_ev]
+    return rq_t, gemm_t
+
+
+def gemm_bytes(M, K, N):
+    """Algorithmic bytes of one GEMM launch: packed codes and scales of both operands, bf16 output."""
+    return (M + N) * K * (0.5 + 1 / 32) + 2 * M * N
+
+
+def kernel_records(shapes, rq_t, gemm_t, peaks, ring, groups):
+    """The roofline records of one workload from its per-shape kernel times.  The GEMM record covers
+    the tensor-bound shapes (M >= 1024; all shapes if there is none); shapes with M <= 128 stream the
+    packed weights once and are reported against the HBM copy bandwidth."""
+    fp4_peak = peaks["bf16_tflops"] * FP4_OVER_BF16
+    fp4_sustained = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    big = [i for i, (M, K, N) in enumerate(shapes) if M >= 1024] or list(range(len(shapes)))
+    small = [i for i, (M, K, N) in enumerate(shapes) if M <= 128 and i not in big]
+    flops = sum(2.0 * shapes[i][0] * shapes[i][1] * shapes[i][2] for i in big)
+    t = sum(gemm_t[i] for i in big) * 1e-3
+    tflops = flops / t / 1e12
+    per_shape = []
+    for i, (M, K, N) in enumerate(shapes):
+        tf = 2.0 * M * K * N / (gemm_t[i] * 1e-3) / 1e12
+        gb = gemm_bytes(M, K, N) / (gemm_t[i] * 1e-3) / 1e9
+        per_shape.append({"MKN": [M, K, N], "gemm_us": round(gemm_t[i] * 1e3, 2), "rq_us": round(rq_t[i] * 1e3, 2),
+                          "gemm_tflops": round(tf, 1), "gemm_frac_of_4x_bf16_burst": round(tf / fp4_peak, 4),
+                          "gemm_gbs": round(gb, 1), "gemm_frac_of_hbm_copy": round(gb / peaks["hbm_gbs"], 4)})
+    roofline = {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": tflops, "peak": fp4_peak,
+                "unit": "TFLOP/s", "frac": tflops / fp4_peak,
+                "peak_source": f"{FP4_OVER_BF16:.0f} x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s)",
+                "frac_of_sustained": tflops / fp4_sustained,
+                "frac_of_nominal_fp4": tflops / NOMINAL_FP4_TFLOPS, "nominal_fp4_tflops": NOMINAL_FP4_TFLOPS,
+                "shapes": [list(shapes[i]) for i in big],
+                "algorithmic_bytes": sum(gemm_bytes(*shapes[i]) for i in big),
+                "timing": f"CUDA events around groups of {ring} back-to-back launches, {groups} groups per shape",
+                "per_shape_us": [round(gemm_t[i] * 1e3, 2) for i in big]}
+    decode = None
+    if small:
+        b = sum(gemm_bytes(*shapes[i]) for i in small)
+        ts = sum(gemm_t[i] for i in small) * 1e-3
+        decode = {"bound": "hbm", "kernel": "gemm_mxfp4_kernel", "achieved": b / ts / 1e9, "peak": peaks["hbm_gbs"],
+                  "unit": "GB/s", "frac": b / ts / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+                  "frac_of_nominal_hbm": b / ts / 1e9 / NOMINAL_HBM_GBS,
+                  "shapes": [list(shapes[i]) for i in small], "algorithmic_bytes": b,
+                  "per_shape_us": [round(gemm_t[i] * 1e3, 2) for i in small]}
+    rq_bytes = sum(M * K * 2.53125 for (M, K, N) in shapes)
+    rq_gbs = rq_bytes / (sum(rq_t) * 1e-3) / 1e9
+    rq = {"bound": "hbm", "kernel": "rotate_quantize_direct_kernel", "achieved": rq_gbs, "peak": peaks["hbm_gbs"],
+          "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+          "frac_of_nominal_hbm": rq_gbs / NOMINAL_HBM_GBS,
+          "per_shape_us": [round(t * 1e3, 2) for t in rq_t]}
+    return roofline, decode, rq, per_shape
+
+
+def block_sweep(bro, synth, peaks, blocks, groups):
+    """cfg4: rotate+quantize of the [16384, 4096] tensor for each rotation size.  Per-size times come
+    from CUDA events around groups of back-to-back launches that cycle through a ring of three inputs
+    (3 x 134 MB > L2), so every launch reads from HBM.  2.53125 algorithmic bytes per element."""
+    import torch
+    cfg = synth.CONFIGS["cfg4"]
+    M, K, _ = cfg["shapes"][0]
+    x0 = synth.activations(M, K, seed=cfg["seed"], recipe=cfg["recipe"]).cuda()
+    ring = 3
+    xs = [x0.roll(7 * r, 0).contiguous() for r in range(ring)]
+    codes = [bro.alloc_codes(M, K) for _ in range(ring)]
+    scales = [bro.alloc_scales(M, K, bro.LAYOUT_GEMM) for _ in range(ring)]
+    for _ in range(3):
+        for b in blocks:
+            bro.rotate_quantize_mxfp4(xs[0], b, codes[0], scales[0], bro.LAYOUT_GEMM)
+    torch.cuda.synchronize()
+    group = 2 * ring
+    evs = {b: [] for b in blocks}
+    torch.cuda._sleep(int(2e7))
+    for gi in range(groups):
+        for b in blocks:
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(group):
+                bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+            c.record()
+            evs[b].append((a, c))
+    torch.cuda.synchronize()
+    bytes_per_launch = M * K * 2.53125
+    per_block = {}
+    for b in blocks:
+        ms = statistics.mean(a.elapsed_time(c) / group for a, c in evs[b])
+        gbs = bytes_per_launch / (ms * 1e-3) / 1e9
+        per_block[str(b if b else K)] = {"us": round(ms * 1e3, 2), "gbs": round(gbs, 1),
+                                         "frac_of_measured_copy": round(gbs / peaks["hbm_gbs"], 4),
+                                         "frac_of_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4)}
+    return {"shape_MK": [M, K], "algorithmic_bytes": bytes_per_launch, "per_block": per_block,
+            "timing": f"CUDA events around groups of {group} back-to-back launches, {groups} groups per size"}, (xs, codes, scales)
+
+
 def run_ours(args):
     import torch
     from paper_2511_04214_b200 import build
@@ -265,143 +493,36 @@ def run_ours(args):
     block = args.block
     peaks = measured_peaks()
 
-    # ---- inputs: a ring of independent activation/output sets so that consecutive steps never
-    # find their inputs in L2 (126 MB).
-    per_step_bytes = sum(M * K * 2 + N * K // 2 + M * N * 2 for (M, K, N) in shapes)
-    ring = max(2, min(8, -(-3 * L2_BYTES // per_step_bytes)))
-    sets = []
-    stream = torch.cuda.current_stream()
-    # --randomised: R_i = diag(s) H / sqrt(block) with a seeded +-1 vector per layer (Sec. 5.1)
-    signs = [synth.rotation_signs(K, seed=cfg["seed"] + idx[j]).to(dev) if args.randomised else None
-             for j, (M, K, N) in enumerate(shapes)]
-    for j, (M, K, N) in enumerate(shapes):
-        i = idx[j]
-        w = synth.weights(N, K, seed=cfg["seed"] + i).to(dev)
-        x0 = synth.activations(M, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
-        ws_bytes = bro.linear_workspace_bytes(M, N, K)
-        per_ring = []
-        for r in range(ring):
-            wcodes = bro.alloc_codes(N, K, dev)
-            wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM, dev)
-            if signs[j] is not None:
-                bro.pack_weights_rs(w, block, signs[j], wcodes, wscales)  # offline, untimed
-            else:
-                bro.pack_weights(w, block, wcodes, wscales)              # offline, untimed
-            x = x0.to(dev).roll(r * 7, 0).contiguous()        # same statistics, separate memory
-            per_ring.append({"x": x, "wcodes": wcodes, "wscales": wscales,
-                             "y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
-                             "ws": bro.alloc_workspace(ws_bytes, dev)})
-        sets.append(per_ring)
-        del w
-    torch.cuda.synchronize()
-
-    def step(r):
-        for i, (M, K, N) in enumerate(shapes):
-            s = sets[i][r % ring]
-            if signs[i] is not None:
-                bro.linear_rs(s["x"], block, signs[i], s["wcodes"], s["wscales"], N, s["y"], s["ws"])
-            else:
-                bro.linear(s["x"], block, s["wcodes"], s["wscales"], N, s["y"], s["ws"])
-
-    flops_per_step = sum(2.0 * M * K * N for (M, K, N) in shapes)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-
-    # ---- warm-up (also sets kernel attributes before any graph capture)
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    torch.cuda.synchronize()
-
-    graph = None
-    if not args.no_graph:
-        # One CUDA graph = `ring` consecutive steps; replayed steps/ring times.
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            for r in range(ring):
-                step(r)
-        graph.replay()
-        torch.cuda.synchronize()
-
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    steps = args.steps
-    if graph is not None:
-        replays = max(1, -(-steps // ring))
-        steps = replays * ring
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.mark("t0")
-    e0.record()
-    if graph is not None:
-        for _ in range(replays):
-            graph.replay()
-    else:
-        for i in range(steps):
-            step(i)
-    e1.record()
-    barrier()
-    sampler.mark("t1")
-    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    layers = Layers(bro, synth, cfg, shapes, idx, block, dev, randomised=args.randomised)
+    ring = layers.ring
+    flops_per_step = layers.flops_per_step()
+
+    ms_local, steps = time_steps(layers, args.steps, args.warmup, not args.no_graph, barrier, sampler)
+    ms_total = max_over_ranks(ms_local, dist, dev)
     status = bro.last_device_status()
     if status != 0:
         raise SystemExit(f"device status {bro.status_string(status)} after the timed region")
     value = aggregate_throughput(flops_per_step, steps, world, ms_total) / 1e12
 
-    # ---- instrumented pass for the per-kernel roofline: the two C-ABI calls bro_linear makes,
-    # each timed with CUDA events around a group of `ring` back-to-back launches (one per ring
-    # set, so no launch finds its operands in L2); per-launch time = group time / ring.  Timing
-    # every launch with its own pair of events adds microseconds of event latency to kernels
-    # that only run for ten.
-    inst_steps = max(3, min(steps // ring, 16))
-    rq_ms = [[] for _ in shapes]
-    gemm_ms = [[] for _ in shapes]
-
-    def views(i, r):
-        M, K, N = shapes[i]
-        s = sets[i][r]
-        nc = bro.codes_bytes(M, K)
-        off = (nc + 1023) // 1024 * 1024
-        return s, s["ws"][:nc], s["ws"][off:off + bro.scales_bytes(M, K, bro.LAYOUT_GEMM)]
-
-    torch.cuda._sleep(int(4e7))        # hold the stream (~20 ms) while the launches below queue up
-    for it in range(inst_steps + 2):
-        for i, (M, K, N) in enumerate(shapes):
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-            ev[0].record()
-            for r in range(ring):
-                s, acodes, ascales = views(i, r)
-                if signs[i] is not None:
-                    bro.rotate_quantize_mxfp4_rs(s["x"], block, signs[i], acodes, ascales, bro.LAYOUT_GEMM)
-                else:
-                    bro.rotate_quantize_mxfp4(s["x"], block, acodes, ascales, bro.LAYOUT_GEMM)
-            ev[1].record()
-            for r in range(ring):
-                s, acodes, ascales = views(i, r)
-                bro.gemm_mxfp4(acodes, ascales, s["wcodes"], s["wscales"], M, N, K, s["y"])
-            ev[2].record()
-            if it >= 2:
-                rq_ms[i].append((ev[0], ev[1]))
-                gemm_ms[i].append((ev[1], ev[2]))
-    torch.cuda.synchronize()
-    rq_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in rq_ms]
-    gemm_t = [statistics.mean(a.elapsed_time(b) for a, b in lst) / ring for lst in gemm_ms]
-    gemm_flops = sum(2.0 * M * K * N for (M, K, N) in shapes)
-    gemm_tflops = gemm_flops / (sum(gemm_t) * 1e-3) / 1e12
-    rq_bytes = sum(M * K * 2.53125 for (M, K, N) in shapes)
-    rq_gbs = rq_bytes / (sum(rq_t) * 1e-3) / 1e9
-    fp4_peak = peaks["bf16_tflops"] * FP4_OVER_BF16
-    gemm_bytes = sum((M + N) * K * (0.5 + 1 / 32) + 2 * M * N for (M, K, N) in shapes)
+    groups = max(3, min(steps // ring, 16))
+    rq_t, gemm_t = time_kernels(layers, groups)
+    roofline, decode, rq_rec, per_shape = kernel_records(shapes, rq_t, gemm_t, peaks, ring, groups)
+    roofline["traffic"] = ncu_traffic(args.workload, [tuple(s) for s in roofline["shapes"]])
 
     # ---- end-to-end through the host-buffer entry point
     e2e = None
     if not args.no_e2e and not args.randomised:     # (the host-buffer entry point has no randomised form)
         host = []
         for i, (M, K, N) in enumerate(shapes):
-            s = sets[i][0]
+            s = layers.sets[i][0]
             host.append({"xh": s["x"].cpu().pin_memory(),
                          "yh": torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
                          "xs": torch.empty((M, K), dtype=torch.bfloat16, device=dev)})
@@ -421,16 +542,19 @@ def run_ours(args):
                 st.wait_event(start)
             for _ in range(n):
                 for i, (M, K, N) in enumerate(shapes):
-                    s, h = sets[i][0], host[i]
+                    s, h = layers.sets[i][0], host[i]
                     bro.linear_host(h["xh"], block, s["wcodes"], s["wscales"], N, h["yh"], h["xs"], s["y"], s["ws"],
                                     stream=lay[i])
             for st in lay:
                 done = torch.cuda.Event()
                 done.record(st)
                 main.wait_event(done)
-        e2e_steps(3)
+        h2d = sum(M * K * 2 for (M, K, N) in shapes)
+        d2h = sum(M * N * 2 for (M, K, N) in shapes)
+        e2e_steps(3 if h2d + d2h < (1 << 30) else 1)
         barrier()
-        n_e2e = max(3, min(steps, 30))
+        # about a second of PCIe traffic at 25 GB/s, at least 3 steps
+        n_e2e = int(max(3, min(steps, 30, 25e9 / max(h2d + d2h, 1))))
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         e2e_steps(n_e2e)
@@ -438,17 +562,52 @@ def run_ours(args):
         barrier()
         ms = max_over_ranks(a.elapsed_time(b), dist, dev)
         e2e = {"value": aggregate_throughput(flops_per_step, n_e2e, world, ms) / 1e12, "unit": UNIT,
-               "h2d_bytes_per_step": sum(M * K * 2 for (M, K, N) in shapes),
-               "d2h_bytes_per_step": sum(M * N * 2 for (M, K, N) in shapes), "steps": n_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": ms / n_e2e,
                "streams": len(shapes)}
-
+        del host
     clocks = sampler.stop() if rank == 0 else None
+    status = bro.last_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {bro.status_string(status)} after the end-to-end region")
+
+    # ---- the other workloads, per kernel, in the same process (rank 0 of a single-GPU run)
+    per_config = None
+    if rank == 0 and world == 1 and not args.no_per_config and args.shape_index < 0:
+        del layers
+        torch.cuda.empty_cache()
+        per_config = {}
+        for name in ("cfg2", "cfg3"):
+            if name == args.workload:
+                continue
+            c2 = synth.CONFIGS[name]
+            sh = [s for s in c2["shapes"] if s[2] > 0]
+            lay2 = Layers(bro, synth, c2, sh, list(range(len(sh))), 32, dev)
+            ms2, st2 = time_steps(lay2, 4 * lay2.ring, 3, True, barrier)
+            g2 = 8
+            rq2, gm2 = time_kernels(lay2, g2)
+            roof2, dec2, rqrec2, ps2 = kernel_records(sh, rq2, gm2, peaks, lay2.ring, g2)
+            per_config[name] = {"value": lay2.flops_per_step() * st2 / (ms2 * 1e-3) / 1e12, "unit": UNIT,
+                                "ms_per_step": ms2 / st2, "steps": st2, "block": 32,
+                                "gemm": {k: roof2[k] for k in ("achieved", "peak", "frac", "frac_of_nominal_fp4", "unit")},
+                                "rotate_quantize": {k: rqrec2[k] for k in ("achieved", "peak", "frac", "frac_of_nominal_hbm", "unit")},
+                                "per_shape": ps2}
+            del lay2
+            torch.cuda.empty_cache()
+        sweep, keep = block_sweep(bro, synth, peaks, synth.CONFIGS["cfg4"]["blocks"], 8)
+        per_config["cfg4"] = sweep
+        del keep
+        torch.cuda.empty_cache()
+        status = bro.last_device_status()
+        if status != 0:
+            raise SystemExit(f"device status {bro.status_string(status)} after the per-config pass")
+    else:
+        del layers
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, single-GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        rows = 256
+        rows = 128
         prepared = oracle_prepare(shapes, cfg, rows, block, idx)
         t, f, passes = 0.0, 0.0, 0
         while t < 10.0 and passes < 200:          # about 10 s of CPU work
@@ -464,26 +623,26 @@ def run_ours(args):
             "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "mxfp4 (e2m1 x e8m0) operands, f32 accumulate, bf16 out", "data": "synthetic",
             "config": {"workload": args.workload, "shapes_MKN": shapes, "block": block,
-                       "l2": f"ring of {ring} independent input/output sets ({per_step_bytes * ring / 1e6:.0f} MB) > 126 MB L2",
-                       "launch": "cuda_graph" if graph is not None else "direct", "parallelism": "replicas only",
+                       "l2": f"ring of {ring} independent input/output sets ({layers_bytes(shapes) * ring / 1e6:.0f} MB) > 126 MB L2",
+                       "launch": "direct" if args.no_graph else "cuda_graph", "parallelism": "replicas only",
                        "rotation": "randomised block Hadamard (diag(s) H)" if args.randomised else "block Hadamard"},
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": steps * len(shapes) * 2,
-            "roofline": {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak,
-                         "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak,
-                         "peak_source": f"{FP4_OVER_BF16:.0f} x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s)",
-                         "traffic": ncu_traffic(args.workload, shapes), "algorithmic_bytes": gemm_bytes,
-                         "timing": f"CUDA events around groups of {ring} back-to-back launches, {inst_steps} groups per shape",
-                         "per_shape_us": [round(t * 1e3, 2) for t in gemm_t]},
-            "rotate_quantize": {"bound": "hbm", "achieved": rq_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                "frac": rq_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                                "per_shape_us": [round(t * 1e3, 2) for t in rq_t]},
+            "roofline": roofline,
+            "decode": decode,
+            "rotate_quantize": rq_rec,
+            "per_shape": per_shape,
+            "per_config": per_config,
             "cpu_baseline": cpu,
         }
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def layers_bytes(shapes):
+    return sum(M * K * 2 + N * K // 2 + M * N * 2 for (M, K, N) in shapes)
 
 
 def run_rotate_quantize_only(args):
@@ -612,13 +771,44 @@ def run_rotate_quantize_only(args):
     print(json.dumps(out), flush=True)
 
 
+def launch_ranks(n, argv):
+    """Start `n` ranks of this script on one node with torch.distributed.run and relay their output
+    (the path does not shard: the ranks are independent replicas that only meet for the timing
+    barrier and the max-over-ranks reduction).  Returns the launcher's exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.run(cmd).returncode
+
+
+def run_rank_check(args):
+    """Host logic of a multi-rank run, without a GPU: every rank reports a rank-dependent time, the
+    job's time is the slowest rank's, rank 0 prints one line.  (Used by the CPU tests to cover the
+    launcher and the rank plumbing with the gloo backend.)"""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = max_over_ranks(10.0 + 5.0 * rank, dist if world > 1 else None, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"rank_check": True, "n_gpus": world, "ms": ms,
+                          "value": aggregate_throughput(1000.0, 4, world, ms)}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--block", type=int, default=32)
     ap.add_argument("--shape-index", type=int, default=-1,
                     help="run only this shape of the workload (for profiling captures); -1 = all")
@@ -630,8 +820,16 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="skip the per-kernel figures of the other workloads (cfg2, cfg3, cfg4)")
+    ap.add_argument("--rank-check", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        # no launcher around us: start the N replica ranks ourselves
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.rank_check:
+        run_rank_check(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.workload == "cfg4":
         run_rotate_quantize_only(args)
