@@ -669,7 +669,7 @@ def run_rotate_quantize_only(args):
     steps = args.steps
     for _ in range(max(args.warmup, 3)):
         for b in blocks:
-            bro.rotate_quantize_mxfp4(xs[0], b, codes[0], scales[0], bro.LAYOUT_GEMM)
+            bro.rotate_quantize_mxfp4(xs[0], b, codes[0], scales[0], bro.LAYOUT_GEMM, flags=args.flags)
     torch.cuda.synchronize()
     sampler.mark("t0")
     t_all0 = torch.cuda.Event(enable_timing=True); t_all1 = torch.cuda.Event(enable_timing=True)
@@ -688,7 +688,7 @@ def run_rotate_quantize_only(args):
             a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for i in range(group):
-                bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+                bro.rotate_quantize_mxfp4(xs[i % ring], b, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM, flags=args.flags)
             c.record()
             evs[b].append((a, c))
     t_all1.record()
@@ -760,7 +760,7 @@ def run_rotate_quantize_only(args):
            "warmup": max(args.warmup, 3), "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16 in, f32 rotation, mxfp4 out", "data": "synthetic",
            "config": {"workload": "cfg4", "shape_MK": [M, K], "blocks": [b if b else K for b in blocks],
-                      "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm"},
+                      "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm", "flags": args.flags},
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
            "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse, "gpu_format_study": format_study,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
@@ -822,6 +822,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the per-kernel figures of the other workloads (cfg2, cfg3, cfg4)")
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0,
+                    help="kernel-selection flags (BRO_FLAG_* of include/bro.h) passed to the *_ex entry points")
     ap.add_argument("--rank-check", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":

@@ -105,6 +105,20 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t shfl_xor2(uint64_t v, int lane_mask) {
+  float lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+  lo = __shfl_xor_sync(0xFFFFFFFFu, lo, lane_mask);
+  hi = __shfl_xor_sync(0xFFFFFFFFu, hi, lane_mask);
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
 
 // 8 bf16 (one 16-byte chunk) -> 4 pairs, fused with butterfly stage h = 1, which pairs the two
 // halves of one 32-bit word: (lo, hi) -> (lo + hi, lo - hi).
@@ -131,6 +145,134 @@ __device__ __forceinline__ void fwht32_stages_2_to_16(uint64_t (&P)[16]) {
       }
     }
   }
+}
+
+// ---- blocks of 64 / 128 channels: cross-lane stages that exchange HALF of each lane's values --------
+// The 2 (or 4) MX groups of a block sit in neighbouring lanes.  A butterfly stage between two lanes
+// needs, for every element i, a + b in one lane and a - b in the other.  Instead of every lane
+// fetching all 32 partner values and producing 32 results, each lane keeps 16 of its values, sends
+// the other 16, and produces BOTH the sum and the difference for the 16 elements it kept: half the
+// shuffles, and the arithmetic stays on packed pairs.  Afterwards a lane holds 16 values of one output
+// group and 16 values of another (two 8-byte code stores instead of one 16-byte store; the group
+// maximum takes one more shuffle).
+//
+// So that both lanes of a pair run the same instructions on the same registers, the odd lane loads
+// its 64 bytes with the two 32-byte halves exchanged (register pair k holds true pair k ^ 8): every
+// lane then keeps registers 0..7 and sends registers 8..15.  Stages h = 1..8 never cross the halves;
+// stage h = 16 does, and is written as two fused multiply-adds with the lane's sign s (+1 even lane,
+// -1 odd lane), which yields a + b and a - b in the registers where this lane expects them:
+//   P'[k]   = s * P[k]   + P[k+8]      P'[k+8] = -s * P[k+8] + P[k]
+// Each is ONE rounding of the exact sum or difference (a product with +-1 is exact), i.e. bit-identical
+// to the add / subtract of the contract, including the sign of an exact zero (x - y == x + (-y)).
+__device__ __forceinline__ void fwht32_stages_2_to_8(uint64_t (&P)[16]) {
+#pragma unroll
+  for (int hp = 1; hp < 8; hp <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if ((k & hp) == 0) {
+        const uint64_t a = P[k], b = P[k + hp];
+        P[k] = add2(a, b);
+        P[k + hp] = sub2(a, b);
+      }
+    }
+  }
+}
+__device__ __forceinline__ void stage16_halves_exchanged(uint64_t (&P)[16], uint64_t s2, uint64_t ns2) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint64_t a = P[k], b = P[k + 8];
+    P[k] = fma2(a, s2, b);
+    P[k + 8] = fma2(b, ns2, a);
+  }
+}
+
+// amax of the 16 values held in 8 pairs (three-input maximum of absolute values, two chains).
+__device__ __forceinline__ float amax_pairs8(const uint64_t (&P)[8]) {
+  float m = 0.f, m2 = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; k += 2) {
+    float lo, hi, lo2, hi2;
+    unpack2(P[k], lo, hi);
+    unpack2(P[k + 1], lo2, hi2);
+    asm("max.abs.f32 %0, %0, %1, %2;" : "+f"(m) : "f"(lo), "f"(hi));
+    asm("max.abs.f32 %0, %0, %1, %2;" : "+f"(m2) : "f"(lo2), "f"(hi2));
+  }
+  return fmaxf(m, m2);
+}
+// Scale byte of a group from its pre-normalisation amax, and the 16 codes of the half group in P
+// (same arithmetic as quantize_group).
+__device__ __forceinline__ uint32_t encode_pairs8(const uint64_t (&P)[8], float amax, uint32_t cbits, uint32_t (&w)[2]) {
+  const float c = __uint_as_float(cbits);
+  const uint32_t ef = __float_as_uint(__fmul_rn(amax, c)) >> 23;
+  const uint32_t s = ef > 2u ? ef - 2u : 0u;
+  float r[16];
+  if (ef >= 27u && ef <= 250u) {
+    const float c2 = __uint_as_float(cbits + ((127u - s) << 23));
+    const uint64_t cc = pack2(c2, c2);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) unpack2(mul2(P[k], cc), r[2 * k], r[2 * k + 1]);
+  } else {
+    const float p2 = __uint_as_float((254u - s) << 23);
+    const uint64_t cc = pack2(c, c), pp = pack2(p2, p2);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) unpack2(mul2(mul2(P[k], cc), pp), r[2 * k], r[2 * k + 1]);
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j)
+    w[j] = pack_e2m1x8(r[8 * j], r[8 * j + 1], r[8 * j + 2], r[8 * j + 3], r[8 * j + 4], r[8 * j + 5],
+                       r[8 * j + 6], r[8 * j + 7]);
+  return s;
+}
+
+// The cross-lane stages of a 64- or 128-channel block on the registers described above, then the
+// quantisation of the two half groups this lane ends up with.
+//   lane & 1   which 16 elements of a group this lane keeps (0: elements 0..15, 1: 16..31)
+//   lane & 2   (blocks of 128) which pair of groups: 0 -> groups 0 / 2 of the block, 1 -> groups 1 / 3
+// Outputs: wx / sx = codes of this lane's 16 elements and scale byte of group X, wy / sy of group Y, with
+//   block 64 : X = group 0, Y = group 1 of the block;   block 128 : X = group (lane>>1)&1, Y = X + 2.
+// P must hold the values after stages h = 1..8 (odd lanes: halves exchanged).
+template <int LOG2B>
+__device__ __forceinline__ void cross_lane_split(uint64_t (&P)[16], int lane, uint32_t cbits, uint32_t (&wx)[2],
+                                                 uint32_t& sx, uint32_t (&wy)[2], uint32_t& sy) {
+  static_assert(LOG2B == 6 || LOG2B == 7, "blocks of 64 or 128 channels");
+  const float s0 = (lane & 1) ? -1.f : 1.f;
+  const uint64_t s0p = pack2(s0, s0), ns0p = pack2(-s0, -s0);
+  stage16_halves_exchanged(P, s0p, ns0p);
+  uint64_t X[8], Y[8];
+  if (LOG2B == 6) {
+    // stage h = 32 with lane ^ 1: kept K = P[0..7], received R = partner's P[8..15] (the same elements)
+    //   even lane: X = K + R, Y = K - R;   odd lane: X = R + K, Y = R - K
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint64_t R = shfl_xor2(P[8 + k], 1);
+      X[k] = add2(P[k], R);
+      Y[k] = fma2(P[k], s0p, mul2(R, ns0p));
+    }
+  } else {
+    // stage h = 32 with lane ^ 1, written so that lanes of the second group pair (lane & 2) get sum and
+    // difference in exchanged registers: they keep the difference and send the sum in stage h = 64.
+    const bool second = (lane & 2) != 0;
+    const float one = 1.f;
+    const uint64_t c1 = second ? s0p : pack2(one, one), c2 = second ? ns0p : pack2(one, one);
+    const uint64_t c3 = second ? pack2(one, one) : s0p, c4 = second ? pack2(one, one) : ns0p;
+    const float s1 = second ? -1.f : 1.f;
+    const uint64_t s1p = pack2(s1, s1), ns1p = pack2(-s1, -s1);
+    uint64_t U[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint64_t R = shfl_xor2(P[8 + k], 1);
+      U[k] = fma2(P[k], c1, mul2(R, c2));            // kept for stage h = 64
+      const uint64_t V = fma2(P[k], c3, mul2(R, c4)); // sent
+      const uint64_t R2 = shfl_xor2(V, 2);
+      X[k] = add2(U[k], R2);
+      Y[k] = fma2(U[k], s1p, mul2(R2, ns1p));
+    }
+  }
+  float mx = amax_pairs8(X), my = amax_pairs8(Y);
+  mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+  my = fmaxf(my, __shfl_xor_sync(0xFFFFFFFFu, my, 1));
+  sx = encode_pairs8(X, mx, cbits, wx);
+  sy = encode_pairs8(Y, my, cbits, wy);
 }
 
 // One butterfly stage across two lanes that hold the low / high half of the pairs.

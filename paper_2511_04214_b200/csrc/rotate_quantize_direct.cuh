@@ -12,7 +12,9 @@
 // every byte twice (TMA write, then the consumers' loads) and all consumer warps wake on the same
 // barrier, which together cost about a third of its run time on a [16384, 4096] tensor; here more
 // warps are resident and they drift apart, so loads, arithmetic and stores of different warps
-// overlap.  Blocks of 64 / 128 channels pair lanes l ^ 1 (and l ^ 2) for their last one / two stages.
+// overlap.  Blocks of 64 / 128 channels pair lanes l ^ 1 (and l ^ 2) for their last one / two stages,
+// each lane exchanging half of its values (rq::cross_lane_split); the per-group error kernels keep the
+// whole group in one lane (rq::cross_lane_stage).
 #pragma once
 
 #include "bro_common.cuh"
@@ -42,8 +44,11 @@ struct Params {
 
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
 // (rq::group_error) — the analysis behind the paper's regular-block / outlier-block comparison.
+#ifndef BRO_RQD_WIDE_BLOCKS
+#define BRO_RQD_WIDE_BLOCKS 3
+#endif
 template <int LOG2B, bool SIGNS, bool STATS>
-__global__ void __launch_bounds__(kThreads, 3) rotate_quantize_direct_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WIDE_BLOCKS : 3) rotate_quantize_direct_kernel(const Params p) {
   const int lane = threadIdx.x & 31;
   const int num_warps = (int)gridDim.x * kWarps;
   const int ng = (int)(p.K >> 5);
@@ -58,16 +63,20 @@ __global__ void __launch_bounds__(kThreads, 3) rotate_quantize_direct_kernel(con
   int row = task / p.chunks_per_row, chunk = task - row * p.chunks_per_row;
   const int step_row = num_warps / p.chunks_per_row, step_chunk = num_warps - step_row * p.chunks_per_row;
 
+  // blocks of 64 / 128 (codes path): odd lanes hold their group with the 32-byte halves exchanged
+  constexpr bool kSplit = LOG2B >= 6 && !STATS;
+  const int hswz = (kSplit && (lane & 1)) ? 2 : 0;
+
   auto load = [&](int r, int c, uint4 (&q)[4]) {
     const int g = c * 32 + lane;
     if (r < p.M && g < ng) {
       const uint4* src = reinterpret_cast<const uint4*>(p.x + (int64_t)r * p.ldx + (int64_t)g * 32);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) q[j] = __ldg(src + j);
+      for (int j = 0; j < 4; ++j) q[j] = __ldg(src + (j ^ hswz));
       if (SIGNS) {
         const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)g * 32);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) q[j] = rq::apply_signs(q[j], __ldg(sp + j));
+        for (int j = 0; j < 4; ++j) q[j] = rq::apply_signs(q[j], __ldg(sp + (j ^ hswz)));
       }
     } else {
 #pragma unroll
@@ -87,11 +96,55 @@ __global__ void __launch_bounds__(kThreads, 3) rotate_quantize_direct_kernel(con
     uint64_t P[16];
 #pragma unroll
     for (int j = 0; j < 4; ++j) rq::unpack_stage1(cur[j], P + 4 * j);
+    const int g = chunk * 32 + lane;
+    const bool live = row < p.M && g < ng;
+    if constexpr (kSplit) {
+      rq::fwht32_stages_2_to_8(P);
+      uint32_t wx[2], wy[2], sx, sy;
+      rq::cross_lane_split<LOG2B>(P, lane, cbits, wx, sx, wy, sy);
+      // the lanes of a block share `live` (K is a multiple of the block); this lane's 16 codes of
+      // group X and of group Y are 8 bytes each, at byte (lane & 1) * 8 of the group's 16
+      const int gb = chunk * 32 + (LOG2B == 6 ? (lane & ~1) : (lane & ~3));
+      const int gx = gb + (LOG2B == 6 ? 0 : ((lane >> 1) & 1));
+      const int gy = gx + (LOG2B == 6 ? 1 : 2);
+      if (live) {
+        uint8_t* rowp = p.codes + (int64_t)row * (p.K >> 1) + (lane & 1) * 8;
+        *reinterpret_cast<uint2*>(rowp + (int64_t)gx * 16) = make_uint2(wx[0], wx[1]);
+        *reinterpret_cast<uint2*>(rowp + (int64_t)gy * 16) = make_uint2(wy[0], wy[1]);
+      }
+      // scale bytes of groups 4j..4j+3 -> one 32-bit word in the lane with lane % 4 == 0
+      uint32_t sb;
+      if (LOG2B == 6) {
+        const uint32_t mine = live ? (sx | (sy << 8)) : 0u;          // groups (2i, 2i+1) of this lane pair
+        sb = mine | (__shfl_xor_sync(0xFFFFFFFFu, mine, 2) << 16);
+      } else {
+        const uint32_t mine = live ? (sx | (sy << 16)) : 0u;         // groups (0, 2) or (1, 3) of the block
+        sb = mine | (__shfl_xor_sync(0xFFFFFFFFu, mine, 2) << 8);
+      }
+      if ((lane & 3) == 0 && g < p.groups_padded) {
+        if (p.layout == BRO_LAYOUT_GEMM) {
+          const int64_t off = ((int64_t)(row >> 7) * p.scale_kblocks + (g >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
+          *reinterpret_cast<uint32_t*>(p.scales + off) = sb;
+        } else if (row < p.M && g < ng) {
+          // (ng is a multiple of 2 or 4 here, so the 4 groups of this word exist whenever g + 4 <= ng)
+          uint8_t* dst = p.scales + (int64_t)row * ng + g;
+          if (g + 4 <= ng && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+            *reinterpret_cast<uint32_t*>(dst) = sb;
+          } else {
+            for (int i = 0; i < 4 && g + i < ng; ++i) dst[i] = (uint8_t)(sb >> (8 * i));
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+      task = ntask;
+      row = nrow;
+      chunk = nchunk;
+      continue;
+    }
     rq::fwht32_stages_2_to_16(P);
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
-    const int g = chunk * 32 + lane;
-    const bool live = row < p.M && g < ng;
     if (STATS) {
       const float e = rq::group_error(P, cbits, p.format);
       if (live) p.mse[(int64_t)row * ng + g] = e;
