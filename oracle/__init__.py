@@ -57,6 +57,12 @@ def lib() -> ctypes.CDLL:
         L.bro_ref_group_mse.argtypes = [p, p, p, i64, i64, p]
         L.bro_ref_fake_quantize.argtypes = [p, i64, i64, ci, p]
         L.bro_ref_fake_quantize.restype = ci
+        L.bro_ref_outlier_groups.argtypes = [p, i64, i64, i64, i64, p, p]
+        L.bro_ref_outlier_groups.restype = ci
+        L.bro_ref_scale_histogram.argtypes = [p, p, i64, p]
+        L.bro_ref_scale_histogram.restype = ci
+        L.bro_ref_scale_inflation.argtypes = [p, p, p, i64, p]
+        L.bro_ref_scale_inflation.restype = ci
         for name in ("rotate_rs", "rotate_quantize_mxfp4_rs", "rotate", "quantize", "decode", "rotate_quantize_mxfp4", "pack_weights",
                      "gemm_mxfp4", "gemm_mxfp4_points", "linear", "group_mse"):
             getattr(L, "bro_ref_" + name).restype = ci
@@ -233,3 +239,43 @@ def group_error(y, fmt) -> np.ndarray:
     y = np.ascontiguousarray(y, dtype=np.float32)
     d = y.astype(np.float64) - fake_quantize(y, fmt)
     return (d * d).reshape(y.shape[0], y.shape[1] // MX_GROUP, MX_GROUP).mean(-1)
+
+
+def group_scale_bytes(x_bits, block: int, signs_bits=None) -> np.ndarray:
+    """E8M0 scale byte of every MX group of x R_block ([M, K/32]); block = 1 is the identity rotation,
+    i.e. the scales of the activations as they are."""
+    _, scales = quantize(rotate(x_bits, block, signs_bits))
+    return scales
+
+
+def outlier_groups(x_bits, top_ppm: int = 1000) -> tuple[np.ndarray, int]:
+    """(mask [M, K/32] uint8, threshold bf16 bits): groups holding one of the top ``top_ppm`` millionths
+    of the entries by absolute value (Sec. 4.2, Fig. 6: the top 0.1 % -> 1000 ppm)."""
+    x = _as_bf16_bits(x_bits)
+    M, K = x.shape
+    mask = np.empty((M, K // MX_GROUP), dtype=np.uint8)
+    t = np.zeros(1, dtype=np.uint16)
+    _check(lib().bro_ref_outlier_groups(_ptr(x), M, K, K, int(top_ppm), _ptr(mask), _ptr(t)), "outlier_groups")
+    return mask, int(t[0])
+
+
+def scale_histogram(scales, mask) -> np.ndarray:
+    """[2, 256] uint64: scale-byte histogram of the regular (row 0) and outlier (row 1) groups."""
+    s = np.ascontiguousarray(scales, dtype=np.uint8).ravel()
+    m = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
+    assert s.shape == m.shape
+    hist = np.empty((2, 256), dtype=np.uint64)
+    _check(lib().bro_ref_scale_histogram(_ptr(s), _ptr(m), s.size, _ptr(hist)), "scale_histogram")
+    return hist
+
+
+def scale_inflation(scales_before, scales_after, mask) -> np.ndarray:
+    """[2, 3] uint64: per class (regular, outlier) the number of groups whose scale byte went down,
+    stayed, went up under the rotation."""
+    b = np.ascontiguousarray(scales_before, dtype=np.uint8).ravel()
+    a = np.ascontiguousarray(scales_after, dtype=np.uint8).ravel()
+    m = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
+    assert a.shape == b.shape == m.shape
+    counts = np.empty((2, 3), dtype=np.uint64)
+    _check(lib().bro_ref_scale_inflation(_ptr(b), _ptr(a), _ptr(m), b.size, _ptr(counts)), "scale_inflation")
+    return counts

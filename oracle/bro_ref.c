@@ -374,3 +374,56 @@ int bro_ref_fake_quantize(const float* y, int64_t rows, int64_t K, int format, d
     }
   return 0;
 }
+
+/* ---- scale statistics (Sec. 4.1 regular / outlier blocks; Sec. 4.2 Fig. 6; App. A.3) ---------------- */
+static int cmp_u16_desc(const void* a, const void* b) {
+  uint16_t x = *(const uint16_t*)a, y = *(const uint16_t*)b;
+  return (x < y) - (x > y);
+}
+
+int bro_ref_outlier_groups(const uint16_t* x, int64_t M, int64_t K, int64_t ldx, int64_t top_ppm,
+                           uint8_t* mask, uint16_t* threshold_bits) {
+  if (!x || !mask) return 1;
+  if (M <= 0 || K <= 0 || K % MX_GROUP != 0 || ldx < K || top_ppm <= 0 || top_ppm > 1000000) return 2;
+  const int64_t n = M * K;
+  /* |x| of a finite bf16 is ordered like its low 15 bits read as an integer */
+  uint16_t* mag = (uint16_t*)malloc((size_t)n * sizeof(uint16_t));
+  if (!mag) return 3;
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K; ++k) mag[m * K + k] = (uint16_t)(x[m * ldx + k] & 0x7FFFu);
+  qsort(mag, (size_t)n, sizeof(uint16_t), cmp_u16_desc);
+  int64_t k = (n * top_ppm + 999999) / 1000000; /* ceil */
+  if (k < 1) k = 1;
+  const uint16_t t = mag[k - 1];
+  free(mag);
+  if (threshold_bits) *threshold_bits = t;
+  const int64_t ng = K / MX_GROUP;
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t g = 0; g < ng; ++g) {
+      uint8_t any = 0;
+      for (int i = 0; i < MX_GROUP; ++i)
+        if ((uint16_t)(x[m * ldx + g * MX_GROUP + i] & 0x7FFFu) >= t) any = 1;
+      mask[m * ng + g] = any;
+    }
+  return 0;
+}
+
+int bro_ref_scale_histogram(const uint8_t* scales, const uint8_t* mask, int64_t n, uint64_t* hist) {
+  if (!scales || !mask || !hist) return 1;
+  if (n < 0) return 2;
+  memset(hist, 0, 2 * 256 * sizeof(uint64_t));
+  for (int64_t i = 0; i < n; ++i) hist[(mask[i] ? 256 : 0) + scales[i]] += 1;
+  return 0;
+}
+
+int bro_ref_scale_inflation(const uint8_t* before, const uint8_t* after, const uint8_t* mask, int64_t n,
+                            uint64_t* counts) {
+  if (!before || !after || !mask || !counts) return 1;
+  if (n < 0) return 2;
+  memset(counts, 0, 6 * sizeof(uint64_t));
+  for (int64_t i = 0; i < n; ++i) {
+    const int j = after[i] < before[i] ? 0 : (after[i] == before[i] ? 1 : 2);
+    counts[(mask[i] ? 3 : 0) + j] += 1;
+  }
+  return 0;
+}

@@ -24,7 +24,9 @@
  * examples, brute-force nearest-grid search, idempotence, integer-matmul special cases,
  * the per-element error bound).  One exception: bro_ref_group_mse's *qualitative ordering*
  * between rotation sizes (Sec. 5.2, Fig. 6/7) is "parity unpinned" — the paper prints figures,
- * not numbers; the MSE arithmetic itself is pinned against a numpy restatement.
+ * not numbers; the MSE arithmetic itself is pinned against a numpy restatement.  The scale
+ * statistics (outlier groups, histograms, inflation counts) are pinned by brute force in numpy,
+ * by conservation (every group is counted once) and by a hand-built row with one outlier channel.
  *
  * Data formats (all host pointers):
  *   bf16 input        : uint16_t, the upper 16 bits of the IEEE fp32 pattern.
@@ -116,6 +118,28 @@ int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scale
  * rounded to nearest-even fp16, clamped to the largest finite fp16; a zero scale gives all zeros).
  * Writes the dequantised values (exact in fp64) to deq[rows, K]. */
 int bro_ref_fake_quantize(const float* y, int64_t rows, int64_t K, int format, double* deq);
+
+/* ---- scale statistics behind the regular-block / outlier-block analysis --------------------------
+ * (Sec. 4.1: blocks are "regular" if they hold no outlier and "outlier blocks" otherwise; Sec. 4.2,
+ * Fig. 6 caption: outliers are the top 0.1 % of the activations by absolute value; App. A.3: most
+ * regular blocks' scales grow under global rotation, block rotation removes most of that growth.)
+ * The "scale" here is the E8M0 byte the MXFP4 quantiser assigns to a group of 32 (bro_ref_quantize);
+ * the scales "before rotation" are those of the rotation with block = 1, which is the identity.
+ *
+ * Outlier groups: with n = M*K entries and k = ceil(n * top_ppm / 1e6) (at least 1), t = the k-th
+ * largest |x|; an entry is an outlier iff |x| >= t (ties at t all count); mask[m, g] = 1 iff group g of
+ * row m holds an outlier.  *threshold_bits receives the bf16 pattern of t. */
+int bro_ref_outlier_groups(const uint16_t* x_bf16, int64_t M, int64_t K, int64_t ldx, int64_t top_ppm,
+                           uint8_t* mask, uint16_t* threshold_bits);
+
+/* hist[c][b] = number of groups of class c (0 regular, 1 outlier, by mask) whose scale byte is b. */
+int bro_ref_scale_histogram(const uint8_t* scales, const uint8_t* mask, int64_t n_groups,
+                            uint64_t* hist /* [2][256] */);
+
+/* counts[c][j]: groups of class c whose scale byte after the rotation is lower (j = 0), equal (1) or
+ * higher (2) than before it. */
+int bro_ref_scale_inflation(const uint8_t* scales_before, const uint8_t* scales_after,
+                            const uint8_t* mask, int64_t n_groups, uint64_t* counts /* [2][3] */);
 
 #ifdef __cplusplus
 }
