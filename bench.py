@@ -700,35 +700,44 @@ def run_rotate_quantize_only(args):
         ts = [a.elapsed_time(c) / group for a, c in evs[b]]
         per_block[str(b if b else K)] = {"us": statistics.mean(ts) * 1e3, "gbs": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9,
                                          "frac_of_measured_copy": bytes_per_launch / (statistics.mean(ts) * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    # The oracle's per-group quantisation error per rotation size (Sec. 4.1 / 4.2, Fig. 6-7), on the
-    # first 512 rows: mean over all MX groups, and split into regular and outlier groups (a group
-    # is an outlier group if it holds one of the top 0.1 % |x| entries of the sample).
+    # The oracle's per-group quantisation error per rotation size (Sec. 4.1 / 4.2, Fig. 6-7) and its scale
+    # statistics (App. A.3), on the first 512 rows: mean error over all MX groups and split into regular
+    # and outlier groups (an outlier group holds one of the top 0.1 % |x| entries of the sample), and the
+    # fraction of regular groups whose E8M0 scale byte rises under each rotation.
     oracle_mse = None
     if not args.no_cpu_baseline:
-        import numpy as np
         import oracle
         rows = 512
         xs_cpu = synth.activations(M, K, seed=cfg["seed"], recipe=cfg["recipe"])[:rows]
         bits = synth.bf16_bits(xs_cpu)
-        absx = np.abs(xs_cpu.float().numpy())
-        thresh = np.quantile(absx, 0.999)
-        outlier = (absx.reshape(rows, K // 32, 32) >= thresh).any(-1)
-        oracle_mse = {"rows": rows, "outlier_group_fraction": float(outlier.mean())}
+        omask, othr = oracle.outlier_groups(bits, 1000)
+        outlier = omask.astype(bool)
+        obefore = oracle.group_scale_bytes(bits, 1)
+        oracle_mse = {"rows": rows, "outlier_group_fraction": float(outlier.mean()), "threshold_bf16_bits": othr}
         for b in blocks:
             y = oracle.rotate(bits, b)
             c, sc = oracle.quantize(y)
             mse = oracle.group_mse(y, c, sc)
+            infl = oracle.scale_inflation(obefore, sc, omask)
             oracle_mse[str(b if b else K)] = {"all": float(mse.mean()), "regular": float(mse[~outlier].mean()),
-                                              "outlier": float(mse[outlier].mean())}
-    # The same statistic over the WHOLE tensor on the GPU (bro_group_quant_error), timed the same way:
-    # 2 bytes read per element, 4 bytes written per group.
+                                              "outlier": float(mse[outlier].mean()),
+                                              "regular_scale_up_fraction": float(infl[0, 2]) / float(infl[0].sum()),
+                                              "outlier_scale_down_fraction": float(infl[1, 0]) / max(float(infl[1].sum()), 1.0)}
+    # The same statistics over the WHOLE tensor on the GPU, all through library calls: outlier groups
+    # (bro_outlier_groups), per-group error (bro_group_quant_error: 2 bytes read per element, 4 bytes
+    # written per group), scale bytes before / after each rotation and the inflation counts.
     gpu_mse = {}
     mse_buf = torch.empty((M, K // 32), dtype=torch.float32, device="cuda")
-    absx0 = xs[0].abs()
-    # outlier groups: hold one of the top 0.1 % |x| entries (threshold from the first 16 M entries)
-    sample = absx0.float().flatten()[: 1 << 24]
-    thresh_gpu = torch.kthvalue(sample, int(sample.numel() * 0.999)).values
-    outlier_gpu = (absx0.view(M, K // 32, 32) >= thresh_gpu).any(-1)
+    gmask = torch.empty((M, K // 32), dtype=torch.uint8, device="cuda")
+    ginfo = torch.zeros(4, dtype=torch.int32, device="cuda")
+    gws = torch.empty(bro.outlier_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    bro.outlier_groups(xs[0], gmask, ginfo, gws, top_ppm=1000)
+    outlier_gpu = gmask.bool()
+    sb_before = torch.empty((M, K // 32), dtype=torch.uint8, device="cuda")
+    sb_after = torch.empty((M, K // 32), dtype=torch.uint8, device="cuda")
+    counts = torch.empty((2, 3), dtype=torch.int64, device="cuda")
+    hist = torch.empty((2, 256), dtype=torch.int64, device="cuda")
+    bro.group_scale_bytes(xs[0], 1, sb_before)
     for b in blocks:
         for i in range(3):
             bro.group_quant_error(xs[i % ring], b, mse_buf)
@@ -738,11 +747,22 @@ def run_rotate_quantize_only(args):
             bro.group_quant_error(xs[i % ring], b, mse_buf)
         c.record()
         bro.group_quant_error(xs[0], b, mse_buf)
+        bro.group_scale_bytes(xs[0], b, sb_after)
+        bro.scale_inflation(sb_before, sb_after, gmask, counts)
+        bro.scale_histogram(sb_after, gmask, hist)
         torch.cuda.synchronize()
+        cn = counts.cpu().numpy().astype(float)
+        hn = hist.cpu().numpy().astype(float)
         us = a.elapsed_time(c) * 1e3 / (2 * ring)
         gpu_mse[str(b if b else K)] = {"us": us, "gbs": M * K * 2.125 / us / 1e3, "all": float(mse_buf.mean()),
                                        "regular": float(mse_buf[~outlier_gpu].mean()),
-                                       "outlier": float(mse_buf[outlier_gpu].mean())}
+                                       "outlier": float(mse_buf[outlier_gpu].mean()),
+                                       "regular_scale_up_fraction": cn[0, 2] / cn[0].sum(),
+                                       "outlier_scale_down_fraction": cn[1, 0] / max(cn[1].sum(), 1.0),
+                                       "mean_scale_byte_regular": float((hn[0] * range(256)).sum() / hn[0].sum()),
+                                       "mean_scale_byte_outlier": float((hn[1] * range(256)).sum() / max(hn[1].sum(), 1.0))}
+    gpu_mse["outlier_group_fraction"] = float(outlier_gpu.float().mean())
+    gpu_mse["threshold_bf16_bits"] = int(ginfo[0])
     # Format study (Sec. 3.2 / Fig. 2-3) on the same tensor: mean group error per 4-bit format for the
     # block-32 and the full-dimension rotation.
     format_study = {}

@@ -201,6 +201,46 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
                                      void* stream);
 
 /*
+ * Scale statistics behind the paper's regular-block / outlier-block argument (Sec. 4.1: "regular
+ * blocks" hold no outlier, "outlier blocks" one or more; Sec. 4.2, Fig. 6 caption: outliers are the
+ * top 0.1 % of the activations by absolute value; App. A.3, Fig. 8-9: under global rotation the scales
+ * of most regular blocks grow, block rotation removes most of that growth).  The "scale" of a group is
+ * the E8M0 byte the MXFP4 quantiser gives it.  All results are integers and exact.
+ *
+ * bro_group_scale_bytes: scales[m, g] (uint8 [M, K/32], dense) = the scale byte of group g of row m of
+ *   x R_block.  block = 1 is the identity rotation — the activations as they are ("before rotation");
+ *   32, 64, 128 and 0 (= K) as in bro_rotate_quantize_mxfp4; signs_bf16 NULL or the +-1 vector.
+ *   Nothing else is written.
+ */
+bro_status bro_group_scale_bytes(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                 const void* signs_bf16, uint8_t* scales, void* stream);
+/*
+ * bro_outlier_groups: with n = M*K entries and k = ceil(n * top_ppm / 1e6) (at least 1; 1000 ppm is the
+ *   paper's 0.1 %), t = the k-th largest |x|; an entry is an outlier iff |x| >= t (ties at t all count).
+ *   mask[m, g] (uint8 [M, K/32]) = 1 iff group g of row m holds an outlier, else 0.
+ *   info       device, 4 x uint32, 16-byte aligned: [0] = the bf16 pattern of t, [1] = 0, [2..3] = k.
+ *   workspace  device, bro_outlier_workspace_bytes() bytes, 16-byte aligned (a histogram of the 32768
+ *              bf16 magnitudes; overwritten).
+ *   Inputs must be finite.
+ */
+size_t bro_outlier_workspace_bytes(void);
+bro_status bro_outlier_groups(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int64_t top_ppm,
+                              uint8_t* mask, uint32_t* info, void* workspace, size_t workspace_bytes,
+                              void* stream);
+/*
+ * bro_scale_histogram: hist (device, uint64 [2][256]) is overwritten with the number of groups of each
+ *   class (row 0 regular, row 1 outlier, by mask) that have each scale byte.
+ * bro_scale_inflation: counts (device, uint64 [2][3]) is overwritten with, per class, the number of
+ *   groups whose scale byte after a rotation is lower / equal / higher than before it — counts[0][2]
+ *   over the number of regular groups is the "fraction of regular blocks whose scale grows".
+ *   scales*, mask: device uint8 [n_groups].
+ */
+bro_status bro_scale_histogram(const uint8_t* scales, const uint8_t* mask, int64_t n_groups,
+                               uint64_t* hist, void* stream);
+bro_status bro_scale_inflation(const uint8_t* scales_before, const uint8_t* scales_after,
+                               const uint8_t* mask, int64_t n_groups, uint64_t* counts, void* stream);
+
+/*
  * ---- tuning and testing -------------------------------------------------------------------------
  * The *_ex entry points are the plain ones plus a `flags` word that forces a kernel variant the
  * library would not pick by itself for this problem (the plain entry points pass 0).  Every variant

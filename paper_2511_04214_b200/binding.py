@@ -28,6 +28,8 @@ EXPORTS = [
     "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt",
     "bro_last_device_status_ex", "bro_selftest_expire_wait",
     "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
+    "bro_group_scale_bytes", "bro_outlier_workspace_bytes", "bro_outlier_groups", "bro_scale_histogram",
+    "bro_scale_inflation",
 ]
 
 # kernel-selection flags of the *_ex entry points (testing and tuning)
@@ -92,6 +94,16 @@ def _load() -> ctypes.CDLL:
     L.bro_group_quant_error_fmt.argtypes = [p, i64, i64, i64, ci, p, ci, p, p]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
+    L.bro_group_scale_bytes.restype = ci
+    L.bro_group_scale_bytes.argtypes = [p, i64, i64, i64, ci, p, p, p]
+    L.bro_outlier_workspace_bytes.restype = sz
+    L.bro_outlier_workspace_bytes.argtypes = []
+    L.bro_outlier_groups.restype = ci
+    L.bro_outlier_groups.argtypes = [p, i64, i64, i64, i64, p, p, p, sz, p]
+    L.bro_scale_histogram.restype = ci
+    L.bro_scale_histogram.argtypes = [p, p, i64, p, p]
+    L.bro_scale_inflation.restype = ci
+    L.bro_scale_inflation.argtypes = [p, p, p, i64, p, p]
     L.bro_last_device_status_ex.restype = ci
     L.bro_last_device_status_ex.argtypes = [p, ctypes.POINTER(ci)]
     L.bro_selftest_expire_wait.restype = ci
@@ -306,3 +318,46 @@ def group_quant_error(x: torch.Tensor, block: int, mse: torch.Tensor, signs: tor
     assert mse.shape == (M, K // 32)
     _check(lib.bro_group_quant_error_fmt(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(mse),
                                          _stream(stream)), "bro_group_quant_error_fmt")
+
+
+def group_scale_bytes(x: torch.Tensor, block: int, scales: torch.Tensor, signs: torch.Tensor = None, stream=None) -> None:
+    """E8M0 byte of every MX group of x R_block into ``scales`` (uint8 [M, K/32]); block = 1: no rotation."""
+    assert x.dtype == torch.bfloat16 and scales.dtype == torch.uint8 and scales.is_contiguous()
+    M, K = x.shape
+    assert scales.shape == (M, K // 32)
+    _check(lib.bro_group_scale_bytes(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), _ptr(scales), _stream(stream)),
+           "bro_group_scale_bytes")
+
+
+def outlier_groups(x: torch.Tensor, mask: torch.Tensor, info: torch.Tensor, workspace: torch.Tensor,
+                   top_ppm: int = 1000, stream=None) -> None:
+    """Groups holding one of the top ``top_ppm`` millionths of |x| -> ``mask`` (uint8 [M, K/32]);
+    ``info`` (int32/uint32 [4] on the device) receives the threshold's bf16 pattern and k."""
+    assert x.dtype == torch.bfloat16 and mask.dtype == torch.uint8 and mask.is_contiguous()
+    M, K = x.shape
+    assert mask.shape == (M, K // 32) and info.numel() >= 4 and info.element_size() == 4
+    _check(lib.bro_outlier_groups(_ptr(x), M, K, _ld(x, K), int(top_ppm), _ptr(mask), _ptr(info), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)), "bro_outlier_groups")
+
+
+def outlier_workspace_bytes() -> int:
+    return int(lib.bro_outlier_workspace_bytes())
+
+
+def scale_histogram(scales: torch.Tensor, mask: torch.Tensor, hist: torch.Tensor, stream=None) -> None:
+    """``hist`` (int64 [2, 256] on the device) <- scale-byte histograms of the regular / outlier groups."""
+    assert scales.dtype == torch.uint8 and mask.dtype == torch.uint8 and hist.dtype == torch.int64
+    assert scales.is_contiguous() and mask.is_contiguous() and hist.is_contiguous() and hist.numel() == 512
+    assert scales.numel() == mask.numel()
+    _check(lib.bro_scale_histogram(_ptr(scales), _ptr(mask), scales.numel(), _ptr(hist), _stream(stream)),
+           "bro_scale_histogram")
+
+
+def scale_inflation(before: torch.Tensor, after: torch.Tensor, mask: torch.Tensor, counts: torch.Tensor,
+                    stream=None) -> None:
+    """``counts`` (int64 [2, 3] on the device) <- per class, groups whose byte went down / stayed / went up."""
+    assert before.dtype == after.dtype == mask.dtype == torch.uint8 and counts.dtype == torch.int64
+    assert before.is_contiguous() and after.is_contiguous() and mask.is_contiguous() and counts.numel() == 6
+    assert before.numel() == after.numel() == mask.numel()
+    _check(lib.bro_scale_inflation(_ptr(before), _ptr(after), _ptr(mask), before.numel(), _ptr(counts),
+                                   _stream(stream)), "bro_scale_inflation")

@@ -12,6 +12,7 @@
 #include "rotate_quantize_direct.cuh"
 #include "gemm_mxfp4.cuh"
 #include "gemm_mxfp4_2cta.cuh"
+#include "scale_stats.cuh"
 
 namespace {
 
@@ -334,7 +335,125 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
   if (B > 128)
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, (int)format, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
   if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
-  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, (int)format, mse, di.sm_count, st);
+  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, (int)format, mse, nullptr, di.sm_count, st);
+}
+
+// ---- scale statistics ----------------------------------------------------------------------------
+bro_status bro_group_scale_bytes(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                 const void* signs_bf16, uint8_t* scales, void* stream) {
+  if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (block != 0 && block != 1 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  const int64_t B = block == 0 ? K : block;
+  if (K % B != 0) return BRO_ERR_SHAPE;
+  if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
+  if (M == 0) return BRO_OK;
+  if (!x_bf16 || !scales) return BRO_ERR_NULL;
+  if (ldx % 8 != 0 || !aligned(x_bf16, 16) || !aligned(signs_bf16, 16)) return BRO_ERR_ALIGN;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (block == 1) {
+    // the identity rotation: a sign flip does not change a magnitude, so the signs play no part
+    const unsigned grid = bro::stats::grid_for(M * (K / 32), 256, di.sm_count, 8);
+    return bro::cuda_ok(bro::launch_kernel(bro::stats::group_scale_bytes_identity, grid, 256, 0, st, 1,
+                                           static_cast<const uint16_t*>(x_bf16), M, K, ldx, scales),
+                        "group_scale_bytes launch")
+               ? BRO_OK
+               : BRO_ERR_CUDA;
+  }
+  if (B > 128)
+    return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, scales, nullptr, bro::rq::kFormatScaleOnly,
+                            BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
+  if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
+  return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16,
+                                bro::rq::kFormatScaleOnly, nullptr, scales, di.sm_count, st);
+}
+
+size_t bro_outlier_workspace_bytes(void) { return bro::stats::kWorkspaceBytes; }
+
+bro_status bro_outlier_groups(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int64_t top_ppm,
+                              uint8_t* mask, uint32_t* info, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+  if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (top_ppm <= 0 || top_ppm > 1000000) return BRO_ERR_SHAPE;
+  if (M == 0) return BRO_OK;
+  if (!x_bf16 || !mask || !info || !workspace) return BRO_ERR_NULL;
+  if (ldx % 8 != 0 || !aligned(x_bf16, 16) || !aligned(info, 16) || !aligned(workspace, 16)) return BRO_ERR_ALIGN;
+  if (workspace_bytes < bro::stats::kWorkspaceBytes) return BRO_ERR_WORKSPACE;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned long long* hist = static_cast<unsigned long long*>(workspace);
+  if (!bro::cuda_ok(cudaMemsetAsync(hist, 0, (size_t)bro::stats::kMagBins * 8, st), "cudaMemsetAsync(histogram)"))
+    return BRO_ERR_CUDA;
+  static bro::DeviceOnce once;
+  const int smem = bro::stats::kMagBins * 4;
+  rc = bro::device_once(once, nullptr, [&](int*) { return set_smem(bro::stats::magnitude_histogram, smem); });
+  if (rc != BRO_OK) return rc;
+  const uint16_t* x = static_cast<const uint16_t*>(x_bf16);
+  const unsigned hgrid = bro::stats::grid_for(M * (K / 8), 512, di.sm_count, 1);
+  if (!bro::cuda_ok(bro::launch_kernel(bro::stats::magnitude_histogram, hgrid, 512, (size_t)smem, st, 1, x, M, K, ldx, hist),
+                    "magnitude_histogram launch"))
+    return BRO_ERR_CUDA;
+  const unsigned long long n = (unsigned long long)M * (unsigned long long)K;
+  unsigned long long k = (n * (unsigned long long)top_ppm + 999999ull) / 1000000ull;
+  if (k < 1) k = 1;
+  if (!bro::cuda_ok(bro::launch_kernel(bro::stats::find_threshold, 1u, 1024u, 0, st, 1,
+                                       static_cast<const unsigned long long*>(hist), k, info),
+                    "find_threshold launch"))
+    return BRO_ERR_CUDA;
+  const unsigned mgrid = bro::stats::grid_for(M * (K / 32), 256, di.sm_count, 8);
+  return bro::cuda_ok(bro::launch_kernel(bro::stats::outlier_group_mask, mgrid, 256, 0, st, 1, x, M, K, ldx,
+                                         static_cast<const uint32_t*>(info), mask),
+                      "outlier_group_mask launch")
+             ? BRO_OK
+             : BRO_ERR_CUDA;
+}
+
+bro_status bro_scale_histogram(const uint8_t* scales, const uint8_t* mask, int64_t n_groups, uint64_t* hist,
+                               void* stream) {
+  if (n_groups < 0) return BRO_ERR_SHAPE;
+  if (!hist) return BRO_ERR_NULL;
+  if (!aligned(hist, 8)) return BRO_ERR_ALIGN;
+  if (n_groups > 0 && (!scales || !mask)) return BRO_ERR_NULL;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!bro::cuda_ok(cudaMemsetAsync(hist, 0, 2 * 256 * sizeof(uint64_t), st), "cudaMemsetAsync(scale histogram)"))
+    return BRO_ERR_CUDA;
+  if (n_groups == 0) return BRO_OK;
+  const unsigned grid = bro::stats::grid_for(n_groups, 256 * 16, di.sm_count, 4);
+  return bro::cuda_ok(bro::launch_kernel(bro::stats::scale_histogram, grid, 256, 0, st, 1, scales, mask, n_groups,
+                                         reinterpret_cast<unsigned long long*>(hist)),
+                      "scale_histogram launch")
+             ? BRO_OK
+             : BRO_ERR_CUDA;
+}
+
+bro_status bro_scale_inflation(const uint8_t* scales_before, const uint8_t* scales_after, const uint8_t* mask,
+                               int64_t n_groups, uint64_t* counts, void* stream) {
+  if (n_groups < 0) return BRO_ERR_SHAPE;
+  if (!counts) return BRO_ERR_NULL;
+  if (!aligned(counts, 8)) return BRO_ERR_ALIGN;
+  if (n_groups > 0 && (!scales_before || !scales_after || !mask)) return BRO_ERR_NULL;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!bro::cuda_ok(cudaMemsetAsync(counts, 0, 6 * sizeof(uint64_t), st), "cudaMemsetAsync(inflation counts)"))
+    return BRO_ERR_CUDA;
+  if (n_groups == 0) return BRO_OK;
+  const unsigned grid = bro::stats::grid_for(n_groups, 256 * 16, di.sm_count, 4);
+  return bro::cuda_ok(bro::launch_kernel(bro::stats::scale_inflation, grid, 256, 0, st, 1, scales_before, scales_after, mask,
+                                         n_groups, reinterpret_cast<unsigned long long*>(counts)),
+                      "scale_inflation launch")
+             ? BRO_OK
+             : BRO_ERR_CUDA;
 }
 
 bro_status bro_group_quant_error(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,

@@ -328,6 +328,23 @@ __device__ __forceinline__ uint32_t quantize_group(const uint64_t (&P)[16], uint
   return s;
 }
 
+// Scale byte only: the E8M0 byte quantize_group would assign to the group held in P.
+constexpr int kFormatScaleOnly = 4;     // `format` value of the analysis kernels that selects this output
+__device__ __forceinline__ uint32_t group_scale_byte(const uint64_t (&P)[16], uint32_t cbits) {
+  float m = 0.f, m2 = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; k += 2) {
+    float lo, hi, lo2, hi2;
+    unpack2(P[k], lo, hi);
+    unpack2(P[k + 1], lo2, hi2);
+    asm("max.abs.f32 %0, %0, %1, %2;" : "+f"(m) : "f"(lo), "f"(hi));
+    asm("max.abs.f32 %0, %0, %1, %2;" : "+f"(m2) : "f"(lo2), "f"(hi2));
+  }
+  m = fmaxf(m, m2);
+  const uint32_t ef = __float_as_uint(__fmul_rn(m, __uint_as_float(cbits))) >> 23;
+  return ef > 2u ? ef - 2u : 0u;
+}
+
 // Quantisation error of one group of 32 (paper Sec. 4.1-4.2: block-level error under the shared
 // scale; Sec. 3.2 / Fig. 2-3 for the formats compared): mean over the group of (y - deq(Q(y)))^2 with
 // y = v * c the rotated values.  `format`: 0 MXFP4 (E2M1, scale 2^E, E = floor(log2 amax) - 2),

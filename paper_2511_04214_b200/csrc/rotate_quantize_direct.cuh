@@ -39,7 +39,8 @@ struct Params {
   int chunks_per_row;           // ceil(groups_padded / 32)
   int total_tasks;              // rows_padded * chunks_per_row; one task = one warp, 32 groups of a row
   float* mse;                   // STATS kernels: [M, K/32] per-group quantisation error instead of codes/scales
-  int format;                   // STATS kernels: which 4-bit format (see rq::group_error)
+  int format;                   // STATS kernels: which 4-bit format (see rq::group_error), or
+                                // rq::kFormatScaleOnly: write the E8M0 byte to scales[M, K/32] and nothing else
 };
 
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
@@ -146,8 +147,13 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
     if (STATS) {
-      const float e = rq::group_error(P, cbits, p.format);
-      if (live) p.mse[(int64_t)row * ng + g] = e;
+      if (p.format == rq::kFormatScaleOnly) {
+        const uint32_t sbyte = rq::group_scale_byte(P, cbits);
+        if (live) p.scales[(int64_t)row * ng + g] = (uint8_t)sbyte;
+      } else {
+        const float e = rq::group_error(P, cbits, p.format);
+        if (live) p.mse[(int64_t)row * ng + g] = e;
+      }
 #pragma unroll
       for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
       task = ntask;
@@ -245,14 +251,15 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int l
   return launch_any<false>(p, log2b, sm_count, st);
 }
 
-// Per-group quantisation error only: mse[M, K/32] (fp32).
+// Per-group quantisation error only: mse[M, K/32] (fp32) — or, with format = rq::kFormatScaleOnly, the
+// per-group scale byte only: scale_bytes[M, K/32].
 inline bro_status launch_stats(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs,
-                               int format, float* mse, int sm_count, cudaStream_t st) {
+                               int format, float* mse, uint8_t* scale_bytes, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M; p.K = K; p.ldx = ldx;
   p.codes = nullptr;
-  p.scales = nullptr;
+  p.scales = scale_bytes;
   p.scale_kblocks = 0;
   p.layout = (int)BRO_LAYOUT_CANONICAL;
   p.signs = static_cast<const uint16_t*>(signs);

@@ -94,6 +94,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
         P[2 * c + 1] = rq::pack2(__fmaf_rn(a2, sgn, o.z), __fmaf_rn(a3, sgn, o.w));
       }
     }
+    if (p.format == rq::kFormatScaleOnly) {   // analysis mode (uniform over the grid): scale byte only
+      const uint32_t sbyte = rq::group_scale_byte(P, cbits);
+      if (live) p.scales[row * (p.K >> 5) + gi] = (uint8_t)sbyte;
+      continue;
+    }
     if (p.mse) {                 // analysis mode (uniform over the grid)
       const float e = rq::group_error(P, cbits, p.format);
       if (live) p.mse[row * (p.K >> 5) + gi] = e;
@@ -136,7 +141,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   int threads = p.threads_per_row < 256 ? 256 : p.threads_per_row;
   p.rows_per_iter = threads / p.threads_per_row;
   const size_t smem = K > 1024 ? (size_t)p.rows_per_iter * K * sizeof(float) : 0;
-  if (layout == BRO_LAYOUT_GEMM && !mse) {
+  if (layout == BRO_LAYOUT_GEMM && !mse && format != rq::kFormatScaleOnly) {
     // padding rows / groups of the tiled scale buffer must read as 0
     const size_t bytes = (size_t)((M + 127) / 128) * (size_t)scale_kblocks * 512;
     if (cudaMemsetAsync(scales, 0, bytes, st) != cudaSuccess) return BRO_ERR_CUDA;
