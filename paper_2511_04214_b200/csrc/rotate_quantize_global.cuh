@@ -120,6 +120,198 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
   }
 }
 
+// ---- K = 2048 / 4096, codes path: the stages above stride 16 through two shared-memory transposes ----
+// A thread always works on 32 values in registers, but on a different set in each of three phases, so
+// that every butterfly stage is register arithmetic (no shuffle in the transform):
+//   phase 1   element bits 0..4  : the thread's 32 consecutive channels (as loaded)
+//   phase 2   element bits 5..9  : 32 channels 32 apart (one column of a 32 x 32 block)
+//   phase 3   element bits 10..  : 2 (K = 2048) or 4 (K = 4096) runs of 16 / 8 consecutive channels, 1024 apart
+// Stage order is still ascending stride with one fp32 rounding per add / subtract, so the result is the
+// same bit for bit.  Between the phases the row passes through shared memory (fp32, K values per row,
+// two buffers so that one barrier per transpose suffices); all accesses are bank-conflict free:
+//   transpose 1  writes 8 x 16 bytes per thread, 16-byte pieces XOR-swizzled with the thread index, and
+//                reads 32 scalars per thread (a warp reads one 128-byte line per instruction);
+//   transpose 2  writes 32 scalars per thread (a warp writes one line per instruction) and reads 8 x 16
+//                bytes, pieces swizzled with bits 3..4 of the piece index.
+// After phase 3 a thread holds 8 (16) consecutive values of 4 (2) MX groups; the group maximum takes two
+// (one) shuffles per group, codes go out as one 32-bit (64-bit) store per group.
+template <int LOG2K, bool SIGNS>
+__global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(const Params p) {
+  static_assert(LOG2K == 11 || LOG2K == 12, "K = 2048 or 4096");
+  constexpr int K = 1 << LOG2K;
+  constexpr int T = K / 32;                   // threads per row
+  constexpr int ROWS = 128 / T;               // rows per pass of the CTA
+  constexpr int HB = LOG2K - 10;              // element bits handled in phase 3
+  constexpr int NJ = 1 << HB;                 // runs per thread in phase 3
+  constexpr int RUN = 32 / NJ;                // consecutive values per run
+  extern __shared__ float xbuf[];             // [2][ROWS][K]
+  constexpr uint32_t cbits = (LOG2K % 2 == 0) ? (uint32_t)(127 - LOG2K / 2) << 23
+                                              : 0x3FB504F3u - ((uint32_t)((LOG2K + 1) / 2) << 23);
+  const int t = threadIdx.x % T;              // thread within the row
+  const int rs = threadIdx.x / T;             // row slot
+  const int lo5 = t & 31, hi = t >> 5;
+  float* bufA = xbuf + (size_t)rs * K;
+  float* bufB = xbuf + (size_t)(ROWS + rs) * K;
+  const int64_t row_iters = (p.M + ROWS - 1) / ROWS;
+
+  griddep_wait();
+  griddep_launch_dependents();
+
+  uint4 sg[4] = {};
+  if (SIGNS) {
+    const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)t * 32);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sg[j] = __ldg(sp + j);
+  }
+  auto load = [&](int64_t it, uint4 (&q)[4]) {
+    const int64_t row = it * ROWS + rs;
+    if (row < p.M) {
+      const uint4* src = reinterpret_cast<const uint4*>(p.x + row * p.ldx + (int64_t)t * 32);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) q[j] = __ldg(src + j);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) q[j] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  // shared-memory addresses that do not change from row to row
+  const uint32_t a_w = smem_u32(bufA) + (uint32_t)t * 128u;                     // transpose 1, writes
+  uint32_t a_r[8];                                                               // transpose 1, reads: row j + 32 hi
+#pragma unroll
+  for (int m = 0; m < 8; ++m)
+    a_r[m] = smem_u32(bufA) + (uint32_t)hi * 4096u + (uint32_t)(((lo5 >> 2) ^ m) << 4) + (uint32_t)((lo5 & 3) << 2);
+  uint32_t b_w[4];                                                               // transpose 2, writes
+#pragma unroll
+  for (int m = 0; m < 4; ++m)
+    b_w[m] = smem_u32(bufB) + (uint32_t)hi * 4096u + (uint32_t)(((lo5 >> 2) ^ m) << 4) + (uint32_t)((lo5 & 3) << 2);
+  const uint32_t b_r = smem_u32(bufB);                                           // transpose 2, reads
+
+  uint4 cur[4], nxt[4];
+  int64_t it = blockIdx.x;
+  if (it < row_iters) load(it, cur);
+  for (; it < row_iters; it += gridDim.x) {
+    if (it + gridDim.x < row_iters) load(it + gridDim.x, nxt);
+    const int64_t row = it * ROWS + rs;
+    const bool live = row < p.M;
+    uint64_t P[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rq::unpack_stage1(SIGNS ? rq::apply_signs(cur[j], sg[j]) : cur[j], P + 4 * j);
+    rq::fwht32_stages_2_to_16(P);                                   // strides 1..16
+    // ---- transpose 1
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      float a0, a1, a2, a3;
+      rq::unpack2(P[2 * c], a0, a1);
+      rq::unpack2(P[2 * c + 1], a2, a3);
+      asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a_w + (uint32_t)((c ^ (t & 7)) << 4)), "f"(a0), "f"(a1),
+                   "f"(a2), "f"(a3)
+                   : "memory");
+    }
+    __syncthreads();
+    {
+      float v[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[j]) : "r"(a_r[j & 7] + (uint32_t)(j * 128)) : "memory");
+      // strides 32..256 on pairs (v[k], v[k + 16]); stride 512 inside the pairs
+#pragma unroll
+      for (int k = 0; k < 16; ++k) P[k] = rq::pack2(v[k], v[k + 16]);
+      rq::fwht32_stages_2_to_16(P);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        float lo, hi2;
+        rq::unpack2(P[k], lo, hi2);
+        v[k] = __fadd_rn(lo, hi2);
+        v[k + 16] = __fsub_rn(lo, hi2);
+      }
+      // ---- transpose 2: value j is element lo5 + 32 j + 1024 hi of the row
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(b_w[j & 3] + (uint32_t)(j * 128)), "f"(v[j]) : "memory");
+    }
+    __syncthreads();
+    // ---- phase 3: runs of RUN consecutive values at RUN * t + 1024 * j2
+    uint64_t E[NJ][RUN / 2];
+#pragma unroll
+    for (int j2 = 0; j2 < NJ; ++j2) {
+#pragma unroll
+      for (int h = 0; h < RUN / 4; ++h) {
+        const uint32_t ci = (uint32_t)(j2 * 256 + t * (RUN / 4) + h);              // 16-byte piece of the row
+        float a0, a1, a2, a3;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(a0), "=f"(a1), "=f"(a2), "=f"(a3)
+                     : "r"(b_r + ((ci ^ ((ci >> 3) & 3u)) << 4))
+                     : "memory");
+        E[j2][2 * h] = rq::pack2(a0, a1);
+        E[j2][2 * h + 1] = rq::pack2(a2, a3);
+      }
+    }
+#pragma unroll
+    for (int hb = 1; hb < NJ; hb <<= 1) {                          // strides 1024 (and 2048)
+#pragma unroll
+      for (int j2 = 0; j2 < NJ; ++j2) {
+        if ((j2 & hb) == 0) {
+#pragma unroll
+          for (int i = 0; i < RUN / 2; ++i) {
+            const uint64_t a = E[j2][i], b = E[j2 + hb][i];
+            E[j2][i] = rq::add2(a, b);
+            E[j2 + hb][i] = rq::sub2(a, b);
+          }
+        }
+      }
+    }
+    // ---- quantise: run j2 belongs to group (t >> HB) + 32 j2; the NJ lanes t, t^1 (, t^2, t^3) share it
+#pragma unroll
+    for (int j2 = 0; j2 < NJ; ++j2) {
+      float m = 0.f;
+#pragma unroll
+      for (int i = 0; i < RUN / 2; ++i) {
+        float lo, hi2;
+        rq::unpack2(E[j2][i], lo, hi2);
+        asm("max.abs.f32 %0, %0, %1, %2;" : "+f"(m) : "f"(lo), "f"(hi2));
+      }
+#pragma unroll
+      for (int d = 1; d < NJ; d <<= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+      const float c = __uint_as_float(cbits);
+      const uint32_t ef = __float_as_uint(__fmul_rn(m, c)) >> 23;
+      const uint32_t sc = ef > 2u ? ef - 2u : 0u;
+      float r[RUN];
+      if (ef >= 27u && ef <= 250u) {
+        const float c2 = __uint_as_float(cbits + ((127u - sc) << 23));
+        const uint64_t cc = rq::pack2(c2, c2);
+#pragma unroll
+        for (int i = 0; i < RUN / 2; ++i) rq::unpack2(rq::mul2(E[j2][i], cc), r[2 * i], r[2 * i + 1]);
+      } else {
+        const float p2 = __uint_as_float((254u - sc) << 23);
+        const uint64_t cc = rq::pack2(c, c), pp = rq::pack2(p2, p2);
+#pragma unroll
+        for (int i = 0; i < RUN / 2; ++i) rq::unpack2(rq::mul2(rq::mul2(E[j2][i], cc), pp), r[2 * i], r[2 * i + 1]);
+      }
+      uint32_t w[RUN / 8];
+#pragma unroll
+      for (int i = 0; i < RUN / 8; ++i)
+        w[i] = rq::pack_e2m1x8(r[8 * i], r[8 * i + 1], r[8 * i + 2], r[8 * i + 3], r[8 * i + 4], r[8 * i + 5], r[8 * i + 6],
+                               r[8 * i + 7]);
+      if (live) {
+        const int g = (t >> HB) + 32 * j2;
+        uint8_t* dst = p.codes + row * (K >> 1) + g * 16 + (t & (NJ - 1)) * (RUN / 2);
+        if (RUN == 8) *reinterpret_cast<uint32_t*>(dst) = w[0];
+        else *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[RUN / 8 - 1]);
+        if ((t & (NJ - 1)) == 0) {
+          if (p.layout == BRO_LAYOUT_GEMM) {
+            const int64_t off = ((row >> 7) * p.scale_kblocks + (g >> 2)) * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4 + (g & 3);
+            p.scales[off] = (uint8_t)sc;
+          } else {
+            p.scales[row * (K >> 5) + g] = (uint8_t)sc;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+  }
+}
+
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
                          void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
   Params p;
@@ -145,6 +337,32 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
     // padding rows / groups of the tiled scale buffer must read as 0
     const size_t bytes = (size_t)((M + 127) / 128) * (size_t)scale_kblocks * 512;
     if (cudaMemsetAsync(scales, 0, bytes, st) != cudaSuccess) return BRO_ERR_CUDA;
+  }
+  if ((K == 2048 || K == 4096) && !mse && format != rq::kFormatScaleOnly) {
+    // codes path at these sizes: all stages in registers, two shared-memory transposes
+    const int rows = (int)(128 / (K / 32));
+    const int64_t iters2 = (M + rows - 1) / rows;
+    const size_t smem2 = (size_t)2 * rows * K * sizeof(float);            // 32 KiB
+    auto go2 = [&](auto kernel) -> bro_status {
+      static DeviceOnce once;                                             // (one per instantiation)
+      int per_sm = 1;
+      const bro_status rc = device_once(once, &per_sm, [&](int* n) {
+        if (!cuda_ok(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2),
+                     "cudaFuncSetAttribute(rotate_quantize_global_smem)"))
+          return BRO_ERR_CUDA;
+        return cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, kernel, 128, smem2),
+                       "occupancy(rotate_quantize_global_smem)")
+                   ? BRO_OK
+                   : BRO_ERR_CUDA;
+      });
+      if (rc != BRO_OK) return rc;
+      const int64_t cap = (int64_t)sm_count * per_sm;
+      const unsigned grid2 = (unsigned)(iters2 < cap ? iters2 : cap);
+      return cuda_ok(launch_kernel(kernel, grid2, 128u, smem2, st, 1, p), "rotate_quantize_global_smem launch") ? BRO_OK
+                                                                                                                 : BRO_ERR_CUDA;
+    };
+    if (K == 4096) return signs ? go2(rotate_quantize_global_smem_kernel<12, true>) : go2(rotate_quantize_global_smem_kernel<12, false>);
+    return signs ? go2(rotate_quantize_global_smem_kernel<11, true>) : go2(rotate_quantize_global_smem_kernel<11, false>);
   }
   const int64_t iters = (M + p.rows_per_iter - 1) / p.rows_per_iter;
   const int64_t max_grid = (int64_t)sm_count * (threads <= 512 ? 2 : 1);
