@@ -124,6 +124,26 @@ bro_status bro::gemm2::make_scale_map(CUtensorMap* map, const void* scales, int6
                      CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
+// Rows of x as a 3-D tensor {64 bf16, K / 64, M} with strides {128 bytes, ldx * 2 bytes}: a box of
+// whole rows lands in shared memory as 128-byte segments with the 128-byte swizzle.
+bro_status bro::rqg::make_row_map(CUtensorMap* map, const void* x, int64_t M, int64_t K, int64_t ldx, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) {
+    snprintf(bro::g_last_cuda_error, sizeof(bro::g_last_cuda_error), "cuTensorMapEncodeTiled unavailable");
+    return BRO_ERR_CUDA;
+  }
+  cuuint64_t dims[3] = {64, (cuuint64_t)(K / 64), (cuuint64_t)M};
+  cuuint64_t strides[2] = {128, (cuuint64_t)ldx * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)(K / 64), (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    snprintf(bro::g_last_cuda_error, sizeof(bro::g_last_cuda_error), "cuTensorMapEncodeTiled (rows): CUresult %d", (int)r);
+  return r == CUDA_SUCCESS ? BRO_OK : BRO_ERR_CUDA;
+}
+
 namespace {
 
 // One warp waits on a barrier that nothing completes: the bounded wait runs out, records its site and

@@ -135,8 +135,13 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
 //                bytes, pieces swizzled with bits 3..4 of the piece index.
 // After phase 3 a thread holds 8 (16) consecutive values of 4 (2) MX groups; the group maximum takes two
 // (one) shuffles per group, codes go out as one 32-bit (64-bit) store per group.
+// The bf16 rows arrive by TMA (one 8 KiB box per pass: ROWS rows x K/64 segments of 128 bytes, 128-byte
+// swizzle), issued by thread 0 for the NEXT pass as soon as every thread has taken its 64 bytes of the
+// current one: the load/store unit's data path, which bounds this kernel, then carries only the
+// conflict-free shared-memory reads instead of one 128-byte line per two lanes of a global load.
 template <int LOG2K, bool SIGNS>
-__global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(const Params p) {
+__global__ void __launch_bounds__(128, 5) rotate_quantize_global_smem_kernel(const __grid_constant__ CUtensorMap tmx,
+                                                                              const Params p) {
   static_assert(LOG2K == 11 || LOG2K == 12, "K = 2048 or 4096");
   constexpr int K = 1 << LOG2K;
   constexpr int T = K / 32;                   // threads per row
@@ -144,7 +149,11 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
   constexpr int HB = LOG2K - 10;              // element bits handled in phase 3
   constexpr int NJ = 1 << HB;                 // runs per thread in phase 3
   constexpr int RUN = 32 / NJ;                // consecutive values per run
-  extern __shared__ float xbuf[];             // [2][ROWS][K]
+  constexpr uint32_t kRawBytes = (uint32_t)ROWS * K * 2;          // 8 KiB
+  extern __shared__ uint8_t smem_raw[];       // [raw bf16 box | barrier | fp32 [2][ROWS][K]], 1 KiB aligned
+  const uint32_t raw = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar = raw + kRawBytes;
+  float* xbuf = reinterpret_cast<float*>(smem_raw + (raw - smem_u32(smem_raw)) + kRawBytes + 1024);
   constexpr uint32_t cbits = (LOG2K % 2 == 0) ? (uint32_t)(127 - LOG2K / 2) << 23
                                               : 0x3FB504F3u - ((uint32_t)((LOG2K + 1) / 2) << 23);
   const int t = threadIdx.x % T;              // thread within the row
@@ -154,8 +163,26 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
   float* bufB = xbuf + (size_t)(ROWS + rs) * K;
   const int64_t row_iters = (p.M + ROWS - 1) / ROWS;
 
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
   griddep_wait();
   griddep_launch_dependents();
+  // this thread's 64 bytes inside the box: segment (t >> 1) of row slot rs, 16-byte pieces 4 (t & 1) + i,
+  // stored at piece index ^ (segment & 7)
+  const uint32_t seg = (uint32_t)rs * (K / 64) + (uint32_t)(t >> 1);
+  const uint32_t raw_mine = raw + seg * 128u;
+  const uint32_t raw_swz = seg & 7u;
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmx);
+    if ((int64_t)blockIdx.x < row_iters) {
+      mbar_arrive_expect_tx(bar, kRawBytes);
+      tma_load_3d(raw, &tmx, 0, 0, (int)((int64_t)blockIdx.x * ROWS), bar);
+    }
+  }
 
   uint4 sg[4] = {};
   if (SIGNS) {
@@ -163,17 +190,6 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
 #pragma unroll
     for (int j = 0; j < 4; ++j) sg[j] = __ldg(sp + j);
   }
-  auto load = [&](int64_t it, uint4 (&q)[4]) {
-    const int64_t row = it * ROWS + rs;
-    if (row < p.M) {
-      const uint4* src = reinterpret_cast<const uint4*>(p.x + row * p.ldx + (int64_t)t * 32);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) q[j] = __ldg(src + j);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) q[j] = make_uint4(0u, 0u, 0u, 0u);
-    }
-  };
   // shared-memory addresses that do not change from row to row
   const uint32_t a_w = smem_u32(bufA) + (uint32_t)t * 128u;                     // transpose 1, writes
   uint32_t a_r[8];                                                               // transpose 1, reads: row j + 32 hi
@@ -186,16 +202,18 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
     b_w[m] = smem_u32(bufB) + (uint32_t)hi * 4096u + (uint32_t)(((lo5 >> 2) ^ m) << 4) + (uint32_t)((lo5 & 3) << 2);
   const uint32_t b_r = smem_u32(bufB);                                           // transpose 2, reads
 
-  uint4 cur[4], nxt[4];
-  int64_t it = blockIdx.x;
-  if (it < row_iters) load(it, cur);
-  for (; it < row_iters; it += gridDim.x) {
-    if (it + gridDim.x < row_iters) load(it + gridDim.x, nxt);
+  uint32_t parity = 0;
+  for (int64_t it = blockIdx.x; it < row_iters; it += gridDim.x) {
     const int64_t row = it * ROWS + rs;
-    const bool live = row < p.M;
+    const bool live = row < p.M;                      // (rows beyond M arrive as zeros)
+    const bool ok = mbar_wait(bar, parity, SITE_RQ_FULL);
+    parity ^= 1u;
     uint64_t P[16];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) rq::unpack_stage1(SIGNS ? rq::apply_signs(cur[j], sg[j]) : cur[j], P + 4 * j);
+    for (int j = 0; j < 4; ++j) {
+      const uint4 q = lds128(raw_mine + ((((uint32_t)(t & 1) * 4u + (uint32_t)j) ^ raw_swz) << 4));
+      rq::unpack_stage1(SIGNS ? rq::apply_signs(q, sg[j]) : q, P + 4 * j);
+    }
     rq::fwht32_stages_2_to_16(P);                                   // strides 1..16
     // ---- transpose 1
 #pragma unroll
@@ -207,7 +225,12 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
                    "f"(a2), "f"(a3)
                    : "memory");
     }
-    __syncthreads();
+    // (also: every thread has taken its bytes of the bf16 box; a lost load ends the loop for all)
+    if (!__syncthreads_and(ok)) break;
+    if (threadIdx.x == 0 && it + gridDim.x < row_iters) {
+      mbar_arrive_expect_tx(bar, kRawBytes);
+      tma_load_3d(raw, &tmx, 0, 0, (int)((it + gridDim.x) * ROWS), bar);
+    }
     {
       float v[32];
 #pragma unroll
@@ -307,10 +330,11 @@ __global__ void __launch_bounds__(128, 6) rotate_quantize_global_smem_kernel(con
         }
       }
     }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
   }
 }
+
+// 3-D view of x for the kernel above: {64 bf16 (128 bytes), K / 64 segments, M rows}, box = whole rows.
+bro_status make_row_map(CUtensorMap* map, const void* x, int64_t M, int64_t K, int64_t ldx, int box_rows);
 
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
                          void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
@@ -342,7 +366,10 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
     // codes path at these sizes: all stages in registers, two shared-memory transposes
     const int rows = (int)(128 / (K / 32));
     const int64_t iters2 = (M + rows - 1) / rows;
-    const size_t smem2 = (size_t)2 * rows * K * sizeof(float);            // 32 KiB
+    const size_t smem2 = (size_t)2 * rows * K * sizeof(float) + (size_t)rows * K * 2 + 2048;   // fp32 buffers, bf16 box, barrier, alignment
+    CUtensorMap tmx;
+    const bro_status mrc = make_row_map(&tmx, x, M, K, ldx, rows);
+    if (mrc != BRO_OK) return mrc;
     auto go2 = [&](auto kernel) -> bro_status {
       static DeviceOnce once;                                             // (one per instantiation)
       int per_sm = 1;
@@ -358,7 +385,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
       if (rc != BRO_OK) return rc;
       const int64_t cap = (int64_t)sm_count * per_sm;
       const unsigned grid2 = (unsigned)(iters2 < cap ? iters2 : cap);
-      return cuda_ok(launch_kernel(kernel, grid2, 128u, smem2, st, 1, p), "rotate_quantize_global_smem launch") ? BRO_OK
+      return cuda_ok(launch_kernel(kernel, grid2, 128u, smem2, st, 1, tmx, p), "rotate_quantize_global_smem launch") ? BRO_OK
                                                                                                                  : BRO_ERR_CUDA;
     };
     if (K == 4096) return signs ? go2(rotate_quantize_global_smem_kernel<12, true>) : go2(rotate_quantize_global_smem_kernel<12, false>);
