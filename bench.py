@@ -56,20 +56,24 @@ def select_shapes(args):
     return cfg, [shapes[i] for i in idx], idx
 
 
-# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch), taken
-# with `ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --clock-control none -k regex:gemm_mxfp4
-# -s 9 -c 3 python bench.py --steps 4 --warmup 3 --no-graph --no-e2e --no-cpu-baseline` (workload cfg2,
-# one value per shape).  The figures belong to one exact version of the kernels: `sources` is the SHA-256
-# over the files of csrc/ at capture time, and the benchmark reports null when they have changed since.
-# (The outputs of these shapes, 8-33 MB, are still dirty in the 126 MB L2 when the kernel ends, which is
-# why the traffic is below the algorithmic bytes.)  "cfg3" holds the one shape captured with `--set full
-# -k regex:gemm_mxfp4 -s 3 -c 2` under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel
-# captured with `-k regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
+# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch) from ncu:
+#   ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum,gpu__time_duration.sum,\
+#       sm__pipe_tensor_cycles_active.avg.pct_of_peak_sustained_elapsed --clock-control none -k regex:gemm_mxfp4 -s 3 -c 2 \
+#       python bench.py --workload cfg5 --shape-index 4 --steps 4 --warmup 3 --no-graph --no-e2e --no-cpu-baseline --no-per-config
+# i.e. ONE shape of the default workload, M = 8192 (K = 8192, N = 28672: 1.6 GB on the device, and a 470 MB
+# output that does not fit the 126 MB L2, so written bytes do reach DRAM).  The traffic of this kernel grows
+# in proportion to M for a fixed weight matrix (the packed weights are re-read once per raster band of 12
+# row tiles, the output is written once), so the figure for the whole record is the captured one scaled by
+# the rows processed.  "cfg3" holds the one shape captured with `--set full -k regex:gemm_mxfp4 -s 3 -c 2`
+# under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel captured with `-k
+# regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
+# The figures belong to one exact version of the kernels: `sources` is the SHA-256 over the files of csrc/
+# at capture time, and the benchmark reports null when they have changed since.
 NCU_TRAFFIC = {
-    "sources": "a56c7b2c27f9fda55cb57728994f0f09dec376166defeab029151a2e894eba40",
-    "cfg2": {(2048, 2048, 2048): 4537344, (2048, 2048, 8192): 11223040, (2048, 8192, 2048): 17906944},
-    "cfg3": {(4096, 4096, 14336): 113546752},
-    "cfg4": {(16384, 4096, 32): 152742400},
+    "sources": "346b1cd6dcacdcac4b8e9b3bc2eed7af9d2fbc2c9f141d25cc2db7dba374760d",
+    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 783179264 + 451448320},
+    "cfg3": {(4096, 4096, 14336): 47678208 + 66902016},
+    "cfg4": {(16384, 4096, 32): 134243328 + 18781440},
 }
 
 
@@ -89,6 +93,12 @@ def ncu_traffic(workload, shapes):
     table = NCU_TRAFFIC.get(workload)
     if table is None or kernel_sources_digest() != NCU_TRAFFIC["sources"]:
         return None
+    if "per_row_of" in table:
+        # one captured shape; the others share its K and N, and traffic grows in proportion to the rows
+        M0, K0, N0 = table["per_row_of"]
+        if any((K, N) != (K0, N0) for (M, K, N) in shapes):
+            return None
+        return float(table["bytes"]) * sum(M for (M, K, N) in shapes) / M0
     try:
         return float(sum(table[tuple(s)] for s in shapes))
     except KeyError:
@@ -516,6 +526,9 @@ def run_ours(args):
     rq_t, gemm_t = time_kernels(layers, groups)
     roofline, decode, rq_rec, per_shape = kernel_records(shapes, rq_t, gemm_t, peaks, ring, groups)
     roofline["traffic"] = ncu_traffic(args.workload, [tuple(s) for s in roofline["shapes"]])
+    if roofline["traffic"] is not None and "per_row_of" in NCU_TRAFFIC.get(args.workload, {}):
+        roofline["traffic_note"] = ("ncu capture of the M = %d shape (%d bytes per launch), scaled by the rows processed"
+                                    % (NCU_TRAFFIC[args.workload]["per_row_of"][0], NCU_TRAFFIC[args.workload]["bytes"]))
 
     # ---- end-to-end through the host-buffer entry point
     e2e = None
