@@ -205,10 +205,16 @@ def oracle_prepare(shapes, cfg, rows_per_shape, block, idx=None):
         i = idx[j] if idx is not None else j
         m = min(M, rows_per_shape)
         x = synth.activations(m, K, seed=cfg["seed"] + i, recipe=cfg["recipe"])
-        w = synth.weights(N, K, seed=cfg["seed"] + i)
-        wc, ws = oracle.pack_weights(synth.bf16_bits(w), block)
+        key = (N, K, cfg["seed"] + i, block)
+        if key not in _PACKED_BY_ORACLE:
+            w = synth.weights(N, K, seed=cfg["seed"] + i)
+            _PACKED_BY_ORACLE[key] = oracle.pack_weights(synth.bf16_bits(w), block)
+        wc, ws = _PACKED_BY_ORACLE[key]
         prepared.append((synth.bf16_bits(x), wc, ws, m, K, N))
     return prepared
+
+
+_PACKED_BY_ORACLE = {}      # offline weight packing by the oracle, done once per weight matrix
 
 
 def oracle_step(prepared, block):
