@@ -39,6 +39,7 @@ FLAG_GEMM_PAIR = 0x10
 FLAG_GEMM_TILE_N128 = 0x20
 FLAG_GEMM_TILE_N256 = 0x40
 FLAG_GEMM_NO_SPLIT = 0x80
+FLAG_GEMM_SINGLE = 0x100
 
 
 class BroError(RuntimeError):

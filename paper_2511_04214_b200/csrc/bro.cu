@@ -511,9 +511,16 @@ static bro_status gemm_impl(const void* acodes, const void* ascales, const void*
   DeviceInfo di;
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
-  // Default: one CTA per 128 x BN tile.  BRO_FLAG_GEMM_PAIR selects the two-CTA kernel (256 x 256
-  // tiles, cta_group::2), which moves a third fewer bytes from L2 but measured no faster.
-  if (flags & BRO_FLAG_GEMM_PAIR)
+  // Two kernels.  The two-CTA kernel (256 x 256 tiles, cta_group::2) moves a third fewer bytes into
+  // shared memory per flop and measures 3-7 % faster once a problem has at least two rounds of
+  // 256 x 256 tiles and tiles long enough (K >= 4096) to amortise its costlier tile hand-over; below
+  // that the single-CTA kernel wins (half-width units for the last round, 128-row granularity, cheaper
+  // prologue).  The flags of the *_ex entry point force either.
+  bool pair = (flags & BRO_FLAG_GEMM_PAIR) != 0;
+  if (!(flags & (BRO_FLAG_GEMM_PAIR | BRO_FLAG_GEMM_SINGLE | BRO_FLAG_GEMM_TILE_N128 | BRO_FLAG_GEMM_TILE_N256 |
+                 BRO_FLAG_GEMM_NO_SPLIT)))
+    pair = K >= 4096 && ceil_div(M, 256) * ceil_div(N, 256) >= 2 * (int64_t)(di.sm_count / 2);
+  if (pair)
     return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, di.sm_count,
                               static_cast<cudaStream_t>(stream));
   return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,

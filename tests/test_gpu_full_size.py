@@ -91,19 +91,20 @@ def test_llm_shaped_layers_full_size(bro, name, index):
     check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, 32, 100000, seed)
 
 
-@pytest.mark.parametrize("variant", ["pair", "tile_n128", "no_split"])
+@pytest.mark.parametrize("variant", ["pair", "single", "tile_n128", "no_split"])
 def test_other_gemm_kernels_on_a_many_tile_shape(bro, variant):
     """M = 4096, K = 4096, N = 14336 (1792 tiles of 128 x 256: twelve per CTA, across raster bands)
-    through the GEMM variants the library does not pick by itself — the two-CTA kernel, 128-column
-    tiles, and the schedule without half-width units — so that their accumulator ping-pong over many
-    tiles per CTA is compared with the oracle too."""
+    through every GEMM variant by flag — the two-CTA kernel (the library's own choice at this size), the
+    single-CTA kernel, 128-column tiles, and the schedule without half-width units — so that each
+    variant's accumulator ping-pong over many tiles per CTA is compared with the oracle."""
     cfg = synth.CONFIGS["cfg3"]
     M, K, N = cfg["shapes"][1]
     seed = synth.config_seed("cfg3", 1)
     x = synth.activations(M, K, seed=seed, recipe=cfg["recipe"])
     w = synth.weights(N, K, seed=seed)
     wc_ref, ws_ref, wcodes, wscales = pack_both(bro, w, 32)
-    flags = {"pair": bro.FLAG_GEMM_PAIR, "tile_n128": bro.FLAG_GEMM_TILE_N128, "no_split": bro.FLAG_GEMM_NO_SPLIT}[variant]
+    flags = {"pair": bro.FLAG_GEMM_PAIR, "single": bro.FLAG_GEMM_SINGLE, "tile_n128": bro.FLAG_GEMM_TILE_N128,
+             "no_split": bro.FLAG_GEMM_NO_SPLIT}[variant]
     check_layer(bro, x, wc_ref, ws_ref, wcodes, wscales, N, 32, 100000, seed, flags=flags)
 
 

@@ -76,13 +76,13 @@ def quantized_pair(M, N, K, seed, block=32, recipe=synth.HEAVY_RECIPE):
     return x, w, ac, asc, wc, wsc
 
 
-@pytest.fixture(params=["default", "cta1_n128", "cta1_n256", "pair"])
+@pytest.fixture(params=["default", "cta1_n128", "cta1_n256", "pair", "single"])
 def tile_n(request, bro):
     """Each GEMM kernel variant in turn, as the `flags` word of bro_gemm_mxfp4_ex: the library's own
     choice, the single-CTA kernel forced to 128- or 256-column tiles, and the two-CTA (cta_group::2)
     kernel with 256 x 256 tiles."""
     return {"default": 0, "cta1_n128": bro.FLAG_GEMM_TILE_N128, "cta1_n256": bro.FLAG_GEMM_TILE_N256,
-            "pair": bro.FLAG_GEMM_PAIR}[request.param]
+            "pair": bro.FLAG_GEMM_PAIR, "single": bro.FLAG_GEMM_SINGLE}[request.param]
 
 
 def test_unit_scales_small_integers_exact(bro, tile_n):
