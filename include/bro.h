@@ -253,7 +253,7 @@ bro_status bro_scale_inflation(const uint8_t* scales_before, const uint8_t* scal
 #define BRO_FLAG_GEMM_PAIR 0x10u      /* GEMM: two CTAs per 256 x 256 tile (cta_group::2) */
 #define BRO_FLAG_GEMM_TILE_N128 0x20u /* GEMM: 128 x 128 tiles */
 #define BRO_FLAG_GEMM_TILE_N256 0x40u /* GEMM: 128 x 256 tiles even when N <= 128 */
-#define BRO_FLAG_GEMM_NO_SPLIT 0x80u  /* GEMM: single-CTA kernel without half-width units in the last round */
+#define BRO_FLAG_GEMM_NO_SPLIT 0x80u  /* GEMM: no half-width units in the last round of the grid */
 #define BRO_FLAG_GEMM_SINGLE 0x100u   /* GEMM: one CTA per 128 x 256 (or 128 x 128) tile, whatever the size */
 bro_status bro_rotate_quantize_mxfp4_ex(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                         const void* signs_bf16, void* codes, void* scales,

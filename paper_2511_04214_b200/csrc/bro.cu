@@ -517,11 +517,10 @@ static bro_status gemm_impl(const void* acodes, const void* ascales, const void*
   // that the single-CTA kernel wins (half-width units for the last round, 128-row granularity, cheaper
   // prologue).  The flags of the *_ex entry point force either.
   bool pair = (flags & BRO_FLAG_GEMM_PAIR) != 0;
-  if (!(flags & (BRO_FLAG_GEMM_PAIR | BRO_FLAG_GEMM_SINGLE | BRO_FLAG_GEMM_TILE_N128 | BRO_FLAG_GEMM_TILE_N256 |
-                 BRO_FLAG_GEMM_NO_SPLIT)))
+  if (!(flags & (BRO_FLAG_GEMM_PAIR | BRO_FLAG_GEMM_SINGLE | BRO_FLAG_GEMM_TILE_N128 | BRO_FLAG_GEMM_TILE_N256)))
     pair = K >= 4096 && ceil_div(M, 256) * ceil_div(N, 256) >= 2 * (int64_t)(di.sm_count / 2);
   if (pair)
-    return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, di.sm_count,
+    return bro::gemm2::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, flags, di.sm_count,
                               static_cast<cudaStream_t>(stream));
   return bro::gemm::launch(acodes, ascales, wcodes, wscales, M, N, K, y, ldy, (int)out_dtype, workspace,
                            workspace_bytes, flags, di.sm_count, static_cast<cudaStream_t>(stream), w_static);

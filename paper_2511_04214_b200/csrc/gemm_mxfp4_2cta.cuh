@@ -53,6 +53,9 @@ struct Params {
   int64_t M, N, ldy;
   int num_k_steps;          // ceil(K/256)
   int tiles_m, tiles_n, total_tiles;   // 256 x 256 tiles
+  // Work units, as in the single-CTA kernel: units [0, full_units) are whole tiles; when the last round
+  // of the grid would be less than half full, its tiles are cut into two 256 x 128 halves each.
+  int full_units, total_units;
 };
 
 // ---- cluster helpers ---------------------------------------------------------------------------
@@ -89,13 +92,24 @@ __device__ __forceinline__ void tma_load_2d_pair_if(uint32_t issue, uint32_t dst
       "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar_cluster), "r"(issue)
       : "memory");
 }
-// E2M1 x E2M1, K-major, UE8M0 scales, M = 256 (128 rows per CTA), N = 256.
+// E2M1 x E2M1, K-major, UE8M0 scales, M = 256 (128 rows per CTA), N = BN.
+template <int BN>
 __device__ __forceinline__ constexpr uint32_t make_idesc_pair() {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | (1u << 23) | ((uint32_t)(256 >> 4) << 24);
+  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(256 >> 4) << 24);
 }
 
 // Tile order: groups of kRasterRows tile rows, column by column inside a group, so that the pairs
 // running at the same time share a few A panels and a few W panels.
+// Unit index -> tile, which half of it (0 when the unit is a whole tile) and its width.
+__device__ __forceinline__ void unit_tile(int u, const Params& p, int& tile, int& half, int& bn) {
+  tile = u; half = 0; bn = kBN;
+  if (u >= p.full_units) {
+    const int idx = u - p.full_units;
+    tile = p.full_units + (idx >> 1);
+    half = idx & 1;
+    bn = kBN / 2;
+  }
+}
 __device__ __forceinline__ void tile_coords(int tile, const Params& p, int& tm, int& tn) {
   const int per_group = kRasterRows * p.tiles_n;
   const int g = tile / per_group;
@@ -108,8 +122,9 @@ __device__ __forceinline__ void tile_coords(int tile, const Params& p, int& tm, 
 template <bool OUT_F32>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_constant__ CUtensorMap tmw,
-                       const __grid_constant__ CUtensorMap tmsfa, const __grid_constant__ CUtensorMap tmsfb,
-                       const __grid_constant__ CUtensorMap tmy, const Params p) {
+                       const __grid_constant__ CUtensorMap tmw_half, const __grid_constant__ CUtensorMap tmsfa,
+                       const __grid_constant__ CUtensorMap tmsfb, const __grid_constant__ CUtensorMap tmy,
+                       const Params p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = smem_base;
@@ -171,24 +186,31 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
         tma_prefetch_desc(&tmw);
         tma_prefetch_desc(&tmsfa);
         tma_prefetch_desc(&tmsfb);
+        if (p.total_units > p.full_units) tma_prefetch_desc(&tmw_half);
       }
       int stage = 0;
       uint32_t phase = 0;
       int64_t issued = 0;
       bool ok = true;
       const uint32_t full0 = map_to_cta(bar_full, 0);      // the leader's barriers, as seen from here
-      for (int tile = pair; tile < p.total_tiles && ok; tile += num_pairs) {
-        int tm, tn;
+      for (int u = pair; u < p.total_units && ok; u += num_pairs) {
+        int tile, half, bn, tm, tn;
+        unit_tile(u, p, tile, half, bn);
         tile_coords(tile, p, tm, tn);
         const int m0 = tm * 256 + (int)rank * kBM;
-        const int n0 = tn * kBN;
+        const int n0 = tn * kBN + half * (kBN / 2);
+        // a half-width unit brings half as many W rows per CTA (through the map with the smaller box)
+        const uint32_t stage_tx = 2u * (uint32_t)(kStageBytes - (bn == kBN ? 0 : kBTileBytes / 2));
         for (int ks = 0; ks < p.num_k_steps; ++ks) {
           if (issued >= kStages) ok = mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, SITE_GEMM_EMPTY);
           if (!ok) break;
-          if (rank == 0) mbar_arrive_expect_tx_if(issue, bar_full + 8 * stage, 2 * kStageBytes);
+          if (rank == 0) mbar_arrive_expect_tx_if(issue, bar_full + 8 * stage, stage_tx);
           const uint32_t full = full0 + 8 * stage;
           tma_load_2d_pair_if(issue, sA + stage * kATileBytes, &tma, ks * 128, m0, full);
-          tma_load_2d_pair_if(issue, sB + stage * kBTileBytes, &tmw, ks * 128, n0 + (int)rank * (kBN / 2), full);
+          if (bn == kBN)
+            tma_load_2d_pair_if(issue, sB + stage * kBTileBytes, &tmw, ks * 128, n0 + (int)rank * (kBN / 2), full);
+          else
+            tma_load_2d_pair_if(issue, sB + stage * kBTileBytes, &tmw_half, ks * 128, n0 + (int)rank * (kBN / 4), full);
           // scale maps are in 32-bit elements: one K step = 1024 bytes = 256 elements per row block
           tma_load_2d_pair_if(issue, sSFA + stage * kSfaBytes, &tmsfa, ks * 256, m0 >> 7, full);
           tma_load_2d_pair_if(issue, sSFB + stage * kSfbBytes, &tmsfb, ks * 256, n0 >> 7, full);
@@ -209,26 +231,38 @@ gemm_mxfp4_pair_kernel(const __grid_constant__ CUtensorMap tma, const __grid_con
     // All 32 lanes of the leader's warp walk the loop together; lane 0 issues for the pair.
     if (rank == 0) {
       const gemm::IssueRing ring = {sA, sB, sSFA, sSFB, bar_full, bar_empty, bar_acc_full, bar_acc_free, bar_ovl_free};
-      const int my_tiles = pair < p.total_tiles ? (p.total_tiles - pair + num_pairs - 1) / num_pairs : 0;
+      auto units_below = [&](int limit) {   // how many of this pair's units have an index below `limit`
+        return pair < limit ? (limit - pair + num_pairs - 1) / num_pairs : 0;
+      };
       gemm::mma_issue_loop<2, kBN, kStages, kATileBytes, kBTileBytes, kSfaBytes, kSfbBytes, kAccStride, true>(
-          ring, tmem_base, tmem_sfa, tmem_sfb, make_idesc_pair(), my_tiles, p.num_k_steps, lane == 0);
+          ring, tmem_base, tmem_sfa, tmem_sfb, make_idesc_pair<kBN>(), units_below(p.total_units), p.num_k_steps,
+          lane == 0, units_below(p.full_units), make_idesc_pair<kBN / 2>());
     }
   } else {
     // ------------------------------ epilogue (both CTAs) ------------------------------
     const int q = warp & 3;
     int it = 0;
-    for (int tile = pair; tile < p.total_tiles; tile += num_pairs, ++it) {
-      int tm, tn;
+    for (int u = pair; u < p.total_units; u += num_pairs, ++it) {
+      int tile, half, bn, tm, tn;
+      unit_tile(u, p, tile, half, bn);
       tile_coords(tile, p, tm, tn);
       const int buf = it & 1;
       if (!mbar_wait_warp(bar_acc_full + 8 * buf, (uint32_t)((it >> 1) & 1), SITE_GEMM_ACC_FULL)) break;
       gemm::tc_fence_after();
       const uint32_t ovl_free_leader = map_to_cta(bar_ovl_free + 8 * buf, 0);
       const uint32_t acc_free_leader = map_to_cta(bar_acc_free + 8 * buf, 0);
-      gemm::epilogue_tile<kChunks, true, OUT_F32>(
-          tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16), buf, lane, tm * 256 + (int)rank * kBM + q * 32,
-          tn * kBN, p.M, p.N, p.y, p.ldy, &tmy, sOut + (uint32_t)q * (32u * 128u), 0u,
-          [&] { mbar_arrive_cluster(ovl_free_leader); }, [&] { mbar_arrive_cluster(acc_free_leader); });
+      const uint32_t tmem_acc = tmem_base + buf * kAccStride + ((uint32_t)(q * 32) << 16);
+      const int row0 = tm * 256 + (int)rank * kBM + q * 32;
+      const int n0 = tn * kBN + half * (kBN / 2);
+      const uint32_t stage_buf = sOut + (uint32_t)q * (32u * 128u);
+      auto release_shared = [&] { mbar_arrive_cluster(ovl_free_leader); };
+      auto release_all = [&] { mbar_arrive_cluster(acc_free_leader); };
+      if (bn == kBN)
+        gemm::epilogue_tile<kChunks, true, OUT_F32>(tmem_acc, buf, lane, row0, n0, p.M, p.N, p.y, p.ldy, &tmy, stage_buf,
+                                                    0u, release_shared, release_all);
+      else
+        gemm::epilogue_tile<kChunks / 2, true, OUT_F32>(tmem_acc, buf, lane, row0, n0, p.M, p.N, p.y, p.ldy, &tmy,
+                                                        stage_buf, 0u, release_shared, release_all);
     }
     // the staging buffer must have been read before this CTA's shared memory goes away; the writes
     // themselves complete with the kernel
@@ -266,8 +300,8 @@ inline int max_resident_pairs(Kern kernel, int sm_count) {
 }
 
 inline bro_status launch(const void* acodes, const void* ascales, const void* wcodes, const void* wscales,
-                         int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, int sm_count,
-                         cudaStream_t st) {
+                         int64_t M, int64_t N, int64_t K, void* y, int64_t ldy, int out_dtype, uint32_t flags,
+                         int sm_count, cudaStream_t st) {
   Params p;
   p.y = y;
   p.M = M; p.N = N; p.ldy = ldy;
@@ -276,12 +310,14 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   p.tiles_m = (int)((M + 255) / 256);
   p.tiles_n = (int)((N + kBN - 1) / kBN);
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
-  if (total > 0x7FFFFFFF) return BRO_ERR_UNSUPPORTED;
+  if (total > 0x3FFFFFFF) return BRO_ERR_UNSUPPORTED;
   p.total_tiles = (int)total;
-  CUtensorMap tma, tmw, tmsfa, tmsfb, tmy;
+  CUtensorMap tma, tmw, tmw_half, tmsfa, tmsfb, tmy;
   bro_status rc = gemm::make_codes_map(&tma, acodes, M, K, kBM);
   if (rc != BRO_OK) return rc;
   rc = gemm::make_codes_map(&tmw, wcodes, N, K, kBN / 2);
+  if (rc != BRO_OK) return rc;
+  rc = gemm::make_codes_map(&tmw_half, wcodes, N, K, kBN / 4);
   if (rc != BRO_OK) return rc;
   rc = make_scale_map(&tmsfa, ascales, M, kblocks, 1);
   if (rc != BRO_OK) return rc;
@@ -293,7 +329,7 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
   } else {
     tmy = tma;   // unused by the fp32-output kernel
   }
-  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, Params),
+  auto go = [&](void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, Params),
                 int which) -> bro_status {
     static DeviceOnce once[2];
     int resident = 0;
@@ -309,9 +345,15 @@ inline bro_status launch(const void* acodes, const void* ascales, const void* wc
       return BRO_OK;
     });
     if (rc != BRO_OK) return rc;
-    const int64_t pairs = total < resident ? total : resident;
-    return cuda_ok(launch_kernel(kernel, (unsigned)(2 * pairs), kThreads, kSmemBytes, st, 2, tma, tmw, tmsfa, tmsfb,
-                                 tmy, p),
+    // Rounds of the persistent grid: when the last round would leave at least half of the pairs idle,
+    // its tiles are cut into two half-width units each (BRO_FLAG_GEMM_NO_SPLIT switches this off).
+    const int64_t rem = total % resident;
+    const bool split = rem > 0 && 2 * rem <= resident && !(flags & BRO_FLAG_GEMM_NO_SPLIT);
+    p.full_units = (int)(split ? total - rem : total);
+    p.total_units = (int)(split ? total + rem : total);
+    const int64_t pairs = p.total_units < resident ? p.total_units : resident;
+    return cuda_ok(launch_kernel(kernel, (unsigned)(2 * pairs), kThreads, kSmemBytes, st, 2, tma, tmw, tmw_half, tmsfa,
+                                 tmsfb, tmy, p),
                    "gemm_mxfp4 pair launch")
                ? BRO_OK
                : BRO_ERR_CUDA;

@@ -129,14 +129,18 @@ def test_ragged_shapes(bro, tile_n, M, N, K):
     run_case(bro, ac, asc, wc, wsc, flags=tile_n)
 
 
-@pytest.mark.parametrize("M,N,K", [(128 * 19, 2048, 256), (128 * 5, 300, 512), (128 * 3, 4 * 256 + 40, 288)])
-def test_half_width_units_of_the_last_round(bro, M, N, K):
-    """Tile counts that leave the last round of the persistent grid less than half full (152 = 148 + 4
-    tiles; 10 and 15 tiles, fewer than half the SMs): the remaining tiles are computed as two
-    half-width units each.  Includes a ragged N whose last half-width unit lies beyond N."""
+@pytest.mark.parametrize("M,N,K", [(128 * 19, 2048, 256), (128 * 5, 300, 512), (128 * 3, 4 * 256 + 40, 288),
+                                   (256 * 19, 1024, 512), (256 * 3, 7 * 256 + 40, 288)])
+@pytest.mark.parametrize("kernel", ["single", "pair"])
+def test_half_width_units_of_the_last_round(bro, kernel, M, N, K):
+    """Tile counts that leave the last round of the persistent grid less than half full (e.g. 152 = 148 + 4
+    tiles of 128 x 256, or 76 = 74 + 2 tiles of 256 x 256 for the two-CTA kernel; 10, 15 and 24 tiles, fewer
+    than half the SMs): the remaining tiles are computed as two half-width units each.  Includes ragged N
+    whose last half-width unit lies beyond N.  With and without the split, in both kernels."""
+    flag = bro.FLAG_GEMM_SINGLE if kernel == "single" else bro.FLAG_GEMM_PAIR
     _, _, ac, asc, wc, wsc = quantized_pair(M, N, K, seed=M + N)
-    run_case(bro, ac, asc, wc, wsc)
-    run_case(bro, ac, asc, wc, wsc, flags=bro.FLAG_GEMM_NO_SPLIT)
+    run_case(bro, ac, asc, wc, wsc, flags=flag)
+    run_case(bro, ac, asc, wc, wsc, flags=flag | bro.FLAG_GEMM_NO_SPLIT)
 
 
 def test_row_stride_of_y(bro, tile_n):
