@@ -62,17 +62,17 @@ def select_shapes(args):
 #       python bench.py --workload cfg5 --shape-index 4 --steps 4 --warmup 3 --no-graph --no-e2e --no-cpu-baseline --no-per-config
 # i.e. ONE shape of the default workload, M = 8192 (K = 8192, N = 28672: 1.6 GB on the device, and a 470 MB
 # output that does not fit the 126 MB L2, so written bytes do reach DRAM).  The traffic of this kernel grows
-# in proportion to M for a fixed weight matrix (the packed weights are re-read once per raster band of 12
-# row tiles, the output is written once), so the figure for the whole record is the captured one scaled by
+# in proportion to M for a fixed weight matrix (the packed weights are re-read once per raster band of 8
+# tile rows of 256, the output is written once), so the figure for the whole record is the captured one scaled by
 # the rows processed.  "cfg3" holds the one shape captured with `--set full -k regex:gemm_mxfp4 -s 3 -c 2`
 # under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel captured with `-k
 # regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
 # The figures belong to one exact version of the kernels: `sources` is the SHA-256 over the files of csrc/
 # at capture time, and the benchmark reports null when they have changed since.
 NCU_TRAFFIC = {
-    "sources": "346b1cd6dcacdcac4b8e9b3bc2eed7af9d2fbc2c9f141d25cc2db7dba374760d",
-    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 783179264 + 451448320},
-    "cfg3": {(4096, 4096, 14336): 47678208 + 66902016},
+    "sources": "fdf508015624d2bbbadbe2ffd6dd31708e35353f6240de08f96cb165ab530527",
+    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 535160064 + 440270336},
+    "cfg3": {(4096, 4096, 14336): 68543744 + 69874944},
     "cfg4": {(16384, 4096, 32): 134243328 + 18781440},
 }
 
@@ -397,6 +397,13 @@ def time_kernels(layers, groups):
     return rq_t, gemm_t
 
 
+def gemm_kernel_name(M, K, N, sm_count=148):
+    """Which GEMM kernel the library picks for this problem (the rule of bro.cu, restated for the record's
+    label; the ncu launch list under profiles/ shows the kernels that actually ran)."""
+    pair = K >= 4096 and (-(-M // 256)) * (-(-N // 256)) >= 2 * (sm_count // 2)
+    return "gemm_mxfp4_pair_kernel" if pair else "gemm_mxfp4_kernel"
+
+
 def gemm_bytes(M, K, N):
     """Algorithmic bytes of one GEMM launch: packed codes and scales of both operands, bf16 output."""
     return (M + N) * K * (0.5 + 1 / 32) + 2 * M * N
@@ -417,10 +424,12 @@ def kernel_records(shapes, rq_t, gemm_t, peaks, ring, groups):
     for i, (M, K, N) in enumerate(shapes):
         tf = 2.0 * M * K * N / (gemm_t[i] * 1e-3) / 1e12
         gb = gemm_bytes(M, K, N) / (gemm_t[i] * 1e-3) / 1e9
-        per_shape.append({"MKN": [M, K, N], "gemm_us": round(gemm_t[i] * 1e3, 2), "rq_us": round(rq_t[i] * 1e3, 2),
+        per_shape.append({"MKN": [M, K, N], "gemm_kernel": gemm_kernel_name(M, K, N),
+                          "gemm_us": round(gemm_t[i] * 1e3, 2), "rq_us": round(rq_t[i] * 1e3, 2),
                           "gemm_tflops": round(tf, 1), "gemm_frac_of_4x_bf16_burst": round(tf / fp4_peak, 4),
                           "gemm_gbs": round(gb, 1), "gemm_frac_of_hbm_copy": round(gb / peaks["hbm_gbs"], 4)})
-    roofline = {"bound": "tensor", "kernel": "gemm_mxfp4_kernel", "achieved": tflops, "peak": fp4_peak,
+    roofline = {"bound": "tensor", "kernel": "/".join(sorted({gemm_kernel_name(*shapes[i]) for i in big})),
+                "achieved": tflops, "peak": fp4_peak,
                 "unit": "TFLOP/s", "frac": tflops / fp4_peak,
                 "peak_source": f"{FP4_OVER_BF16:.0f} x {peaks['source']} bf16 burst ({peaks['bf16_tflops']} TFLOP/s)",
                 "frac_of_sustained": tflops / fp4_sustained,
