@@ -153,6 +153,36 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
                       int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Packed weights with a descriptor.  bro_pack_weights writes two bare buffers; nothing in them says
+ * which rotation they were packed with, so bro_linear cannot notice weights packed with another block
+ * size or sign vector (the rotation would no longer cancel, Eq. 1, and the layer would silently
+ * compute something else).  A caller who wants that check keeps this HOST-side descriptor with the
+ * buffers (and stores it as the header of a weight file): bro_pack_weights_desc fills it,
+ * bro_linear_packed refuses (BRO_ERR_SHAPE) activations whose K, block or use of a sign vector differ,
+ * and a descriptor with the wrong magic or layout version (BRO_ERR_UNSUPPORTED).
+ *   signs_bf16  NULL for the plain rotation, else the +-1 vector (see the randomised forms below).
+ * All other arguments, requirements and errors are those of bro_pack_weights(_rs) / bro_linear(_rs).
+ */
+#define BRO_WEIGHTS_MAGIC 0x344F5242u /* "BRO4" */
+#define BRO_WEIGHTS_VERSION 1u        /* codes row-major [N, K/2]; scales in BRO_LAYOUT_GEMM */
+typedef struct {
+  uint32_t magic;     /* BRO_WEIGHTS_MAGIC */
+  uint32_t version;   /* BRO_WEIGHTS_VERSION */
+  int64_t N, K;
+  int32_t block;      /* rotation block the weights were packed with: 32, 64, 128 or 0 (= K) */
+  int32_t randomised; /* 1 if a sign vector was applied */
+  const void* codes;  /* device, bro_codes_bytes(N, K) bytes */
+  const void* scales; /* device, bro_scales_bytes(N, K, BRO_LAYOUT_GEMM) bytes */
+} bro_packed_weights;
+bro_status bro_pack_weights_desc(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                                 const void* signs_bf16, void* wcodes, void* wscales,
+                                 bro_packed_weights* desc /* host, out */, void* stream);
+bro_status bro_linear_packed(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                             const void* signs_bf16, const bro_packed_weights* weights /* host */,
+                             void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
  * Randomised block rotation (Sec. 5.1, "block-wise randomized Hadamard rotations"): the same three
  * operations with R_i = diag(s) H_block / sqrt(block), s a vector of +-1 over the K channels, i.e.
  * channel k of every row is multiplied by s_k (exactly, a sign-bit flip) before the transform.

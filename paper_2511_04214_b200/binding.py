@@ -29,8 +29,15 @@ EXPORTS = [
     "bro_last_device_status_ex", "bro_selftest_expire_wait",
     "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
     "bro_group_scale_bytes", "bro_outlier_workspace_bytes", "bro_outlier_groups", "bro_scale_histogram",
-    "bro_scale_inflation",
+    "bro_scale_inflation", "bro_pack_weights_desc", "bro_linear_packed",
 ]
+
+
+class PackedWeights(ctypes.Structure):
+    """Host-side descriptor of packed weights (bro_packed_weights of include/bro.h)."""
+    _fields_ = [("magic", ctypes.c_uint32), ("version", ctypes.c_uint32), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("block", ctypes.c_int32), ("randomised", ctypes.c_int32), ("codes", ctypes.c_void_p),
+                ("scales", ctypes.c_void_p)]
 
 # kernel-selection flags of the *_ex entry points (testing and tuning)
 FLAG_RQ_TMA_RING = 0x1
@@ -105,6 +112,10 @@ def _load() -> ctypes.CDLL:
     L.bro_scale_histogram.argtypes = [p, p, i64, p, p]
     L.bro_scale_inflation.restype = ci
     L.bro_scale_inflation.argtypes = [p, p, p, i64, p, p]
+    L.bro_pack_weights_desc.restype = ci
+    L.bro_pack_weights_desc.argtypes = [p, i64, i64, i64, ci, p, p, p, ctypes.POINTER(PackedWeights), p]
+    L.bro_linear_packed.restype = ci
+    L.bro_linear_packed.argtypes = [p, i64, i64, i64, ci, p, ctypes.POINTER(PackedWeights), p, i64, p, sz, p]
     L.bro_last_device_status_ex.restype = ci
     L.bro_last_device_status_ex.argtypes = [p, ctypes.POINTER(ci)]
     L.bro_selftest_expire_wait.restype = ci
@@ -362,3 +373,23 @@ def scale_inflation(before: torch.Tensor, after: torch.Tensor, mask: torch.Tenso
     assert before.numel() == after.numel() == mask.numel()
     _check(lib.bro_scale_inflation(_ptr(before), _ptr(after), _ptr(mask), before.numel(), _ptr(counts),
                                    _stream(stream)), "bro_scale_inflation")
+
+
+def pack_weights_desc(w: torch.Tensor, block: int, wcodes, wscales, signs: torch.Tensor = None, stream=None) -> PackedWeights:
+    """pack_weights that also returns the host-side descriptor (N, K, block, randomised, buffers)."""
+    assert w.dtype == torch.bfloat16 and w.dim() == 2 and w.stride(1) == 1
+    N, K = w.shape
+    desc = PackedWeights()
+    _check(lib.bro_pack_weights_desc(_ptr(w), N, K, _ld(w, K), block, _ptr(signs), _ptr(wcodes), _ptr(wscales),
+                                     ctypes.byref(desc), _stream(stream)), "bro_pack_weights_desc")
+    return desc
+
+
+def linear_packed(x: torch.Tensor, block: int, weights: PackedWeights, y: torch.Tensor, workspace: torch.Tensor,
+                  signs: torch.Tensor = None, stream=None) -> None:
+    """linear that first checks the descriptor against K, block and the use of a sign vector."""
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+    M, K = x.shape
+    _check(lib.bro_linear_packed(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), ctypes.byref(weights), _ptr(y),
+                                 _ld(y, weights.N), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "bro_linear_packed")

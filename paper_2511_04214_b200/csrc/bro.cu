@@ -585,6 +585,37 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
                      workspace_bytes, 0u, stream);
 }
 
+bro_status bro_pack_weights_desc(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,
+                                 const void* signs_bf16, void* wcodes, void* wscales, bro_packed_weights* desc,
+                                 void* stream) {
+  if (!desc) return BRO_ERR_NULL;
+  desc->magic = 0;          // stays invalid unless the packing was enqueued
+  const bro_status rc = launch_rotate_quantize(w_bf16, N, K, ldw, block, signs_bf16, wcodes, wscales, BRO_LAYOUT_GEMM, 0u,
+                                               static_cast<cudaStream_t>(stream));
+  if (rc != BRO_OK) return rc;
+  desc->magic = BRO_WEIGHTS_MAGIC;
+  desc->version = BRO_WEIGHTS_VERSION;
+  desc->N = N;
+  desc->K = K;
+  desc->block = block;
+  desc->randomised = signs_bf16 ? 1 : 0;
+  desc->codes = wcodes;
+  desc->scales = wscales;
+  return BRO_OK;
+}
+
+bro_status bro_linear_packed(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block, const void* signs_bf16,
+                             const bro_packed_weights* weights, void* y_bf16, int64_t ldy, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  if (!weights) return BRO_ERR_NULL;
+  if (weights->magic != BRO_WEIGHTS_MAGIC || weights->version != BRO_WEIGHTS_VERSION) return BRO_ERR_UNSUPPORTED;
+  // the rotation only cancels, (x R)(W R)^T = x W^T, when both sides used the same R
+  if (weights->K != K || weights->block != block || (weights->randomised != 0) != (signs_bf16 != nullptr))
+    return BRO_ERR_SHAPE;
+  return linear_impl(x_bf16, M, K, ldx, block, signs_bf16, weights->codes, weights->scales, weights->N, y_bf16, ldy,
+                     workspace, workspace_bytes, 0u, stream);
+}
+
 bro_status bro_linear_host(const void* x_host_bf16, int64_t M, int64_t K, int block, const void* wcodes,
                            const void* wscales, int64_t N, void* y_host_bf16, void* x_stage, void* y_stage,
                            void* workspace, size_t workspace_bytes, void* stream) {

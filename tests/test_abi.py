@@ -93,3 +93,31 @@ def test_argument_validation_needs_no_device(lib):
     assert L.bro_gemm_mxfp4(p(a128 + 16), p(a128), p(a128), p(a128), 1, 8, 32, p(a128), 8, 0, None, 0, None) == 3
     assert L.bro_gemm_mxfp4(p(a128), p(a128), p(a128), p(a128), 0, 8, 32, p(a128), 8, 0, None, 0, None) == 0
     assert L.bro_linear(p(a128), 4, 32, 32, 32, p(a128), p(a128), 8, p(a128), 8, None, 0, None) == 1
+
+
+def test_packed_weight_descriptor_is_checked_before_any_device_work(lib):
+    """bro_linear_packed refuses weights packed with another block size, another K, with / without a sign
+    vector, or a descriptor that is not one — all on the host, before any CUDA call."""
+    L = lib.lib
+    buf = (ctypes.c_uint8 * 4096)()
+    a = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+    p = ctypes.c_void_p
+    d = lib.PackedWeights(magic=0x344F5242, version=1, N=8, K=64, block=32, randomised=0, codes=a, scales=a)
+    ref = ctypes.byref(d)
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 64, None, ref, p(a), 8, p(a), 1 << 20, None) == 2      # block differs
+    assert L.bro_linear_packed(p(a), 4, 128, 128, 32, None, ref, p(a), 8, p(a), 1 << 20, None) == 2    # K differs
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 32, p(a), ref, p(a), 8, p(a), 1 << 20, None) == 2      # signs on one side only
+    d.randomised = 1
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 32, None, ref, p(a), 8, p(a), 1 << 20, None) == 2
+    d.randomised = 0
+    d.version = 7
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 32, None, ref, p(a), 8, p(a), 1 << 20, None) == 4      # unknown layout version
+    d.version, d.magic = 1, 0
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 32, None, ref, p(a), 8, p(a), 1 << 20, None) == 4      # not a descriptor
+    assert L.bro_linear_packed(p(a), 4, 64, 64, 32, None, None, p(a), 8, p(a), 1 << 20, None) == 1
+    d.magic = 0x344F5242
+    assert L.bro_linear_packed(p(a), 0, 64, 64, 32, None, ref, p(a), 8, p(a), 1 << 20, None) == 0      # M == 0: nothing to do
+    # a failed packing leaves the descriptor invalid
+    out = lib.PackedWeights(magic=0x344F5242)
+    assert L.bro_pack_weights_desc(p(a), 8, 48, 48, 32, None, p(a), p(a), ctypes.byref(out), None) == 2
+    assert out.magic == 0

@@ -91,3 +91,32 @@ def test_whole_layer_with_randomised_rotation(bro, block):
     exact = x.double().numpy() @ w.double().numpy().T
     rel = np.linalg.norm(got - exact) / np.linalg.norm(exact)
     assert rel < 0.25
+
+
+def test_packed_weight_descriptor_round_trip_and_mismatch(bro):
+    """bro_pack_weights_desc / bro_linear_packed: the same bits as bro_linear(_rs) when the descriptor
+    matches, BRO_ERR_SHAPE when the activations ask for another rotation than the weights carry."""
+    M, K, N = 130, 512, 264
+    x = synth.activations(M, K, seed=31).cuda()
+    w = synth.weights(N, K, seed=32).cuda()
+    signs = synth.rotation_signs(K, seed=33).cuda()
+    ws = bro.alloc_workspace(bro.linear_workspace_bytes(M, N, K))
+    for s in (None, signs):
+        wcodes = bro.alloc_codes(N, K); wscales = bro.alloc_scales(N, K, bro.LAYOUT_GEMM)
+        desc = bro.pack_weights_desc(w, 64, wcodes, wscales, signs=s)
+        assert (desc.N, desc.K, desc.block, desc.randomised) == (N, K, 64, 0 if s is None else 1)
+        y1 = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        y2 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        if s is None:
+            bro.linear(x, 64, wcodes, wscales, N, y1, ws)
+        else:
+            bro.linear_rs(x, 64, s, wcodes, wscales, N, y1, ws)
+        bro.linear_packed(x, 64, desc, y2, ws, signs=s)
+        assert bro.last_device_status() == 0
+        assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+        with pytest.raises(bro.BroError) as e:
+            bro.linear_packed(x, 32, desc, y2, ws, signs=s)              # another block size
+        assert e.value.code == 2
+        with pytest.raises(bro.BroError) as e:
+            bro.linear_packed(x, 64, desc, y2, ws, signs=(signs if s is None else None))
+        assert e.value.code == 2
