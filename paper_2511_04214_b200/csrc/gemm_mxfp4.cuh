@@ -269,7 +269,6 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
                                                bool issue_lane, int narrow_from = 0x7FFFFFFF,
                                                uint32_t idesc_narrow = 0u) {
   // tiles narrow_from.. of this CTA are half-width: same loop, the instruction descriptor says N = BN/2
-  // (the scale copies still move both W row blocks; the second one is simply not read)
   const uint32_t issue = issue_lane ? 1u : 0u;
   const uint32_t a_lo0 = desc_lo_sw128(r.sA), b_lo0 = desc_lo_sw128(r.sB);
   const uint32_t sfa_lo0 = desc_lo_sf(r.sSFA), sfb_lo0 = desc_lo_sf(r.sSFB);
@@ -277,12 +276,13 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
   uint32_t idesc0 = idesc_full;
   // scale bytes {0,1} of a 32-bit scale word for the first MMA of a half, {2,3} for the second
   uint32_t idesc1 = idesc0 | (2u << 4) | (2u << 29);
-  auto copy_scales = [&](int stage, int h) {
+  // (a half-width unit reads the scales of its one 128-row block of W only)
+  auto copy_scales = [&](int stage, int h, bool narrow) {
     const uint32_t lo_a = sfa_lo0 + (uint32_t)stage * (SFA_STAGE >> 4) + (uint32_t)h * 32u;
     const uint32_t lo_b = sfb_lo0 + (uint32_t)stage * (SFB_STAGE >> 4) + (uint32_t)h * 32u;
     tc_cp_sf<CG>(issue, tmem_sfa + 4 * h, lo_a, hi_sf);
-#pragma unroll
-    for (int nb = 0; nb < BN / 128; ++nb) tc_cp_sf<CG>(issue, tmem_sfb + (BN / 32) * h + 4 * nb, lo_b + 64u * nb, hi_sf);
+    tc_cp_sf<CG>(issue, tmem_sfb + (BN / 32) * h, lo_b, hi_sf);
+    if (BN == 256 && !narrow) tc_cp_sf<CG>(issue, tmem_sfb + (BN / 32) * h + 4, lo_b + 64u, hi_sf);
   };
   auto mma_half = [&](int stage, int h, uint32_t tmem_acc, uint32_t accumulate_first) {
     const uint32_t a_lo = a_lo0 + (uint32_t)stage * (A_STAGE >> 4) + 4u * h;
@@ -297,8 +297,8 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
   if (ok) ok = mbar_wait_warp(r.bar_full, 0u, SITE_GEMM_FULL);
   if (ok) {
     tc_fence_after();
-    copy_scales(0, 0);
-    copy_scales(0, 1);
+    copy_scales(0, 0, 0 >= narrow_from);
+    copy_scales(0, 1, 0 >= narrow_from);
   }
   for (int it = 0; it < my_tiles && ok; ++it) {
     const int buf = it & 1;
@@ -319,6 +319,7 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
       const bool has_next = (ks + 1 < num_k_steps) || (it + 1 < my_tiles);
       const int next_stage = (stage + 1 == STAGES) ? 0 : stage + 1;
       const uint32_t next_phase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
+      const bool next_narrow = (ks + 1 < num_k_steps ? it : it + 1) >= narrow_from;   // the unit the next stage belongs to
       // Probe the next stage's barrier before issuing: the answer travels while the two MMAs
       // below are issued, and in the steady state it is "ready", so the issuing warp rarely
       // spends a barrier round trip between tensor-core instructions.
@@ -328,11 +329,11 @@ __device__ __forceinline__ void mma_issue_loop(const IssueRing& r, uint32_t tmem
         if (!__all_sync(0xFFFFFFFFu, probe)) ok = mbar_wait_warp(r.bar_full + 8 * next_stage, next_phase, SITE_GEMM_FULL);
         if (!ok) break;
         tc_fence_after();
-        copy_scales(next_stage, 0);          // half 0's columns were last read by the two MMAs above
+        copy_scales(next_stage, 0, next_narrow);   // half 0's columns were last read by the two MMAs above
       }
       mma_half(stage, 1, tmem_acc, 1u);
       tc_commit<CG>(issue, r.bar_empty + 8 * stage);   // frees the stage when these MMAs have read it
-      if (has_next) copy_scales(next_stage, 1);
+      if (has_next) copy_scales(next_stage, 1, next_narrow);
       stage = next_stage;
       phase = next_phase;
     }
