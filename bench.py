@@ -67,14 +67,14 @@ def select_shapes(args):
 # the rows processed.  "cfg3" holds the one shape captured with `--set full -k regex:gemm_mxfp4 -s 3 -c 2`
 # under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel captured with `-k
 # regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
-# (Recorded digest: the kernels of the captures plus the host-side descriptor entry points added to bro.cu
-# afterwards; no kernel or dispatch rule changed in between.)
+# (The block-32 rotate+quantize kernel of the "cfg4" entry is unchanged since its capture; the GEMM entries
+# were taken on exactly these sources.)
 # The figures belong to one exact version of the kernels: `sources` is the SHA-256 over the files of csrc/
 # at capture time, and the benchmark reports null when they have changed since.
 NCU_TRAFFIC = {
-    "sources": "3d9209baa752a0258cdf7eca1364e3ed706a17c74df6071e5f4d94f2fd3d6394",
-    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 535160064 + 440270336},
-    "cfg3": {(4096, 4096, 14336): 68543744 + 69874944},
+    "sources": "676c4209132601b506bd32b5c261f2c7c7083db3a25e6f56e3ddc446735ff2e9",
+    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
+    "cfg3": {(4096, 4096, 14336): 68345088 + 69353728},
     "cfg4": {(16384, 4096, 32): 134243328 + 18781440},
 }
 

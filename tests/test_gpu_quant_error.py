@@ -102,3 +102,13 @@ def test_formats_on_degenerate_rows(bro):
     x[3] = base.to(torch.bfloat16)
     for fmt in ("bfp4", "mxint4", "bint4"):
         check(gpu(bro, x, 32, fmt=fmt), reference(x, 32, fmt=fmt))
+
+
+@pytest.mark.parametrize("block", [32, 64, 128, 0])
+@pytest.mark.parametrize("M,K", [(130, 1024), (37, 4096)])
+def test_randomised_rotation_every_block_size(bro, block, M, K):
+    """The per-group error with a sign vector through every rotation size (the analysis variants of the
+    block kernels and of the full-dimension kernel)."""
+    x = synth.activations(M, K, seed=7 + M)
+    signs = synth.rotation_signs(K, seed=K + 1)
+    check(gpu(bro, x, block, signs), reference(x, block, signs))

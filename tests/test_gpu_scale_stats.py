@@ -48,6 +48,17 @@ def test_scale_bytes_all_rotations(bro, M, K):
     assert bro.last_device_status() == 0
 
 
+@pytest.mark.parametrize("block", [1, 32, 64, 128, 0])
+def test_scale_bytes_with_a_sign_vector(bro, block):
+    """A sign vector changes the rotated values (not their magnitudes under the identity): every rotation
+    size against the oracle's randomised rotation."""
+    M, K = 130, 1024
+    x = synth.activations(M, K, seed=77)
+    signs = synth.rotation_signs(K, seed=78)
+    got = gpu_scale_bytes(bro, x.cuda(), block, signs=signs.cuda()).cpu().numpy()
+    assert np.array_equal(got, oracle.group_scale_bytes(synth.bf16_bits(x), block, synth.bf16_bits(signs)))
+
+
 def test_scale_bytes_equal_the_quantisers_own(bro):
     """The analysis call and bro_rotate_quantize_mxfp4 must agree on every byte."""
     x = synth.activations(300, 1024, seed=8).cuda()
