@@ -68,11 +68,15 @@ def test_random_case(bro, seed):
     ld32 = (N + 3) // 4 * 4          # rows of the output start on 16-byte boundaries
     y32buf = torch.full((M, ld32), float("nan"), dtype=torch.float32, device="cuda")
     y32 = y32buf[:, :N]
-    bro.gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y32)
-    assert bro.last_device_status() == 0
-    got32 = y32.cpu().numpy().astype(np.float64)
-    assert not np.isnan(got32).any()
-    assert np.all(np.abs(got32 - y_ref) <= 1e-5 * S + 1e-6)
+    for flags in (0, bro.FLAG_GEMM_PAIR, bro.FLAG_GEMM_TILE_N128):      # the library's choice, then the other kernels
+        y32buf.fill_(float("nan"))
+        bro.gemm_mxfp4(acodes, ascales, wcodes, wscales, M, N, K, y32, flags=flags)
+        assert bro.last_device_status() == 0
+        got32 = y32.cpu().numpy().astype(np.float64)
+        assert not np.isnan(got32).any()
+        assert np.all(np.abs(got32 - y_ref) <= 1e-5 * S + 1e-6), hex(flags)
+        if ld32 > N:
+            assert torch.isnan(y32buf[:, N:]).all()
 
     # whole layer, bf16 output (a row pitch that keeps rows 16-byte aligned)
     ldy = (N + 7) // 8 * 8
