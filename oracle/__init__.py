@@ -57,6 +57,12 @@ def lib() -> ctypes.CDLL:
         L.bro_ref_group_mse.argtypes = [p, p, p, i64, i64, p]
         L.bro_ref_fake_quantize.argtypes = [p, i64, i64, ci, p]
         L.bro_ref_fake_quantize.restype = ci
+        L.bro_ref_swiglu_f32.argtypes = [p, p, i64, p]
+        L.bro_ref_swiglu_f32.restype = ci
+        L.bro_ref_swiglu.argtypes = [p, p, i64, i64, i64, i64, p]
+        L.bro_ref_swiglu.restype = ci
+        L.bro_ref_swiglu_rotate_quantize_mxfp4.argtypes = [p, p, i64, i64, i64, i64, ci, p, p, p]
+        L.bro_ref_swiglu_rotate_quantize_mxfp4.restype = ci
         L.bro_ref_outlier_groups.argtypes = [p, i64, i64, i64, i64, p, p]
         L.bro_ref_outlier_groups.restype = ci
         L.bro_ref_scale_histogram.argtypes = [p, p, i64, p]
@@ -279,3 +285,39 @@ def scale_inflation(scales_before, scales_after, mask) -> np.ndarray:
     counts = np.empty((2, 3), dtype=np.uint64)
     _check(lib().bro_ref_scale_inflation(_ptr(b), _ptr(a), _ptr(m), b.size, _ptr(counts)), "scale_inflation")
     return counts
+
+
+def swiglu_f32(gate_bits, up_bits) -> np.ndarray:
+    """fp32 value of silu(gate) * up before the bf16 rounding (the fixed fp32 operation sequence)."""
+    g = np.ascontiguousarray(gate_bits, dtype=np.uint16).ravel()
+    u = np.ascontiguousarray(up_bits, dtype=np.uint16).ravel()
+    assert g.shape == u.shape
+    out = np.empty(g.shape, dtype=np.float32)
+    _check(lib().bro_ref_swiglu_f32(_ptr(g), _ptr(u), g.size, _ptr(out)), "swiglu_f32")
+    return out
+
+
+def swiglu(gate_bits, up_bits) -> np.ndarray:
+    """h = bf16(silu(gate) * up) as uint16 bit patterns [M, K]: the input of down_proj, which the online
+    rotation acts on (Sec. 4.3)."""
+    g = _as_bf16_bits(gate_bits)
+    u = _as_bf16_bits(up_bits)
+    assert g.shape == u.shape
+    M, K = g.shape
+    h = np.empty((M, K), dtype=np.uint16)
+    _check(lib().bro_ref_swiglu(_ptr(g), _ptr(u), M, K, K, K, _ptr(h)), "swiglu")
+    return h
+
+
+def swiglu_rotate_quantize_mxfp4(gate_bits, up_bits, block: int, signs_bits=None) -> tuple[np.ndarray, np.ndarray]:
+    g = _as_bf16_bits(gate_bits)
+    u = _as_bf16_bits(up_bits)
+    assert g.shape == u.shape
+    M, K = g.shape
+    codes = np.empty((M, K // 2), dtype=np.uint8)
+    scales = np.empty((M, K // MX_GROUP), dtype=np.uint8)
+    s = _signs(signs_bits, K)
+    _check(lib().bro_ref_swiglu_rotate_quantize_mxfp4(_ptr(g), _ptr(u), M, K, K, K, int(block),
+                                                      None if s is None else _ptr(s), _ptr(codes), _ptr(scales)),
+           "swiglu_rotate_quantize_mxfp4")
+    return codes, scales

@@ -427,3 +427,74 @@ int bro_ref_scale_inflation(const uint8_t* before, const uint8_t* after, const u
   }
   return 0;
 }
+
+/* ---- gated MLP activation feeding the online rotation (Sec. 4.3, the R_4 site before down_proj) ------- */
+static inline float f32_from_bits(uint32_t u) {
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+static inline float silu_mul_f32(float g, float u) {
+  const float LOG2E = f32_from_bits(0x3FB8AA3Bu);  /* fp32(log2 e) */
+  const float LN2_HI = f32_from_bits(0x3F317218u); /* fp32(ln 2) */
+  const float LN2_LO = f32_from_bits(0xB102E308u); /* fp32(ln 2 - LN2_HI) = -1.9046543e-9 */
+  const float t = -fabsf(g);
+  float e = 0.0f;
+  if (t >= -86.0f) {
+    const float n = rintf(t * LOG2E); /* round to nearest, ties to even */
+    float r = fmaf(n, -LN2_HI, t);
+    r = fmaf(n, -LN2_LO, r);
+    float p = f32_from_bits(0x3AB60B61u);        /* 1/720 */
+    p = fmaf(p, r, f32_from_bits(0x3C088889u));  /* 1/120 */
+    p = fmaf(p, r, f32_from_bits(0x3D2AAAABu));  /* 1/24 */
+    p = fmaf(p, r, f32_from_bits(0x3E2AAAABu));  /* 1/6 */
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    /* p in [0.70, 1.42], n in [-124, 0]: scaling by 2^n is an exponent-field addition, exact */
+    e = f32_from_bits(f32_bits(p) + ((uint32_t)(int32_t)n << 23));
+  }
+  const float d = 1.0f + e;
+  const float num = (g >= 0.0f) ? 1.0f : e;
+  const float s = num / d;
+  const float a = g * s;
+  return a * u;
+}
+
+static inline uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u = f32_bits(f);
+  /* finite inputs: add half an ulp of bf16 minus one, plus the lowest kept bit (ties to even) */
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+int bro_ref_swiglu_f32(const uint16_t* gate, const uint16_t* up, int64_t n, float* h32) {
+  if (!gate || !up || !h32) return 1;
+  if (n < 0) return 2;
+  for (int64_t i = 0; i < n; ++i) h32[i] = silu_mul_f32(bf16_to_f32(gate[i]), bf16_to_f32(up[i]));
+  return 0;
+}
+
+int bro_ref_swiglu(const uint16_t* gate, const uint16_t* up, int64_t M, int64_t K, int64_t ldg, int64_t ldu,
+                   uint16_t* h) {
+  if (!gate || !up || !h) return 1;
+  if (M < 0 || K <= 0 || ldg < K || ldu < K) return 2;
+#pragma omp parallel for schedule(static)
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t k = 0; k < K; ++k)
+      h[m * K + k] = f32_to_bf16_rne(silu_mul_f32(bf16_to_f32(gate[m * ldg + k]), bf16_to_f32(up[m * ldu + k])));
+  return 0;
+}
+
+int bro_ref_swiglu_rotate_quantize_mxfp4(const uint16_t* gate, const uint16_t* up, int64_t M, int64_t K,
+                                         int64_t ldg, int64_t ldu, int block, const uint16_t* signs,
+                                         uint8_t* codes, uint8_t* scales) {
+  if (M < 0 || K <= 0) return 2;
+  uint16_t* h = (uint16_t*)malloc((size_t)(M > 0 ? M : 1) * (size_t)K * sizeof(uint16_t));
+  if (!h) return 3;
+  int rc = bro_ref_swiglu(gate, up, M, K, ldg, ldu, h);
+  if (rc == 0) rc = bro_ref_rotate_quantize_mxfp4_rs(h, M, K, K, block, signs, codes, scales);
+  free(h);
+  return rc;
+}

@@ -141,6 +141,24 @@ int bro_ref_scale_histogram(const uint8_t* scales, const uint8_t* mask, int64_t 
 int bro_ref_scale_inflation(const uint8_t* scales_before, const uint8_t* scales_after,
                             const uint8_t* mask, int64_t n_groups, uint64_t* counts /* [2][3] */);
 
+/* ---- the producer of the online-rotated activations -----------------------------------------------
+ * The one rotation paid at inference sits directly before down_proj (Sec. 4.3 "Reduced online
+ * computing"; Sec. 6), whose input in the LLaMA-family models the paper evaluates is the gated MLP
+ * activation h = silu(gate) * up.  The paper does not spell that producer out; this build's reading, in
+ * fp32 with every operation one IEEE round-to-nearest step so that two implementations agree bit for bit:
+ *   t = -|g|;  e = exp(t) as  n = rint(t * log2e), r = fma(n, -ln2_hi, t), r = fma(n, -ln2_lo, r),
+ *   p = 1 + r (1 + r (1/2 + r (1/6 + r (1/24 + r (1/120 + r / 720))))) by Horner with fma, e = p * 2^n
+ *   (e = 0 for t < -86);  sigmoid = (g >= 0 ? 1 : e) / (1 + e);  h = bf16_rne((g * sigmoid) * u).
+ * Pinned against the exact function (|error| of the fp32 value <= 4e-7 relative + 4e-36 |u|), special values,
+ * and an independent bf16 rounding (torch). */
+int bro_ref_swiglu_f32(const uint16_t* gate_bf16, const uint16_t* up_bf16, int64_t n, float* h32);
+int bro_ref_swiglu(const uint16_t* gate_bf16, const uint16_t* up_bf16, int64_t M, int64_t K, int64_t ldg,
+                   int64_t ldu, uint16_t* h_bf16 /* [M, K] dense */);
+/* h as above, then the activation path (rotate + MXFP4 quantise) on it. */
+int bro_ref_swiglu_rotate_quantize_mxfp4(const uint16_t* gate_bf16, const uint16_t* up_bf16, int64_t M,
+                                         int64_t K, int64_t ldg, int64_t ldu, int block,
+                                         const uint16_t* signs_bf16, uint8_t* codes, uint8_t* scales);
+
 #ifdef __cplusplus
 }
 #endif
