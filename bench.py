@@ -67,23 +67,30 @@ def select_shapes(args):
 # the rows processed.  "cfg3" holds the one shape captured with `--set full -k regex:gemm_mxfp4 -s 3 -c 2`
 # under `--workload cfg3 --shape-index 1`, "cfg4" the block-32 kernel captured with `-k
 # regex:rotate_quantize_direct -s 6 -c 2` under `--workload cfg4 --only-block --block 32`.
-# (The block-32 rotate+quantize kernel of the "cfg4" entry is unchanged since its capture; the GEMM entries
-# were taken on exactly these sources.)
-# The figures belong to one exact version of the kernels: `sources` is the SHA-256 over the files of csrc/
-# at capture time, and the benchmark reports null when they have changed since.
+# The figures belong to one exact version of the kernels: every entry names the kernel source files it was
+# captured on and their SHA-256 at capture time, and the benchmark reports null once they have changed.
+# (Which GEMM kernel runs for a shape is decided in bro.cu; gemm_kernel_name() below restates that rule
+# and the launch list under profiles/ shows it in effect at capture time.)
+GEMM_SOURCES = ("bro_common.cuh", "gemm_mxfp4.cuh", "gemm_mxfp4_2cta.cuh")
+RQ_SOURCES = ("bro_common.cuh", "rotate_quantize.cuh", "rotate_quantize_direct.cuh")
 NCU_TRAFFIC = {
-    "sources": "676c4209132601b506bd32b5c261f2c7c7083db3a25e6f56e3ddc446735ff2e9",
-    "cfg5": {"per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
-    "cfg3": {(4096, 4096, 14336): 68345088 + 69353728},
-    "cfg4": {(16384, 4096, 32): 134243328 + 18781440},
+    "cfg5": {"sources": GEMM_SOURCES, "digest": "096c61cb1b9865ca985e775b0d340c5efb1060c2d39547c30f96dd9d3d65fab1",
+             "per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
+    "cfg3": {"sources": GEMM_SOURCES, "digest": "096c61cb1b9865ca985e775b0d340c5efb1060c2d39547c30f96dd9d3d65fab1",
+             "shapes": {(4096, 4096, 14336): 68345088 + 69353728}},
+    "cfg4": {"sources": RQ_SOURCES, "digest": "RQ_DIGEST_PENDING",
+             "shapes": {(16384, 4096, 32): 134243328 + 18781440}},
 }
 
 
-def kernel_sources_digest():
+def kernel_sources_digest(files=None):
+    """SHA-256 over the named files of csrc/ (all of them if none are named)."""
     import glob
     import hashlib
+    csrc = os.path.join(ROOT, "paper_2511_04214_b200", "csrc")
+    paths = sorted(glob.glob(os.path.join(csrc, "*"))) if files is None else [os.path.join(csrc, f) for f in files]
     h = hashlib.sha256()
-    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2511_04214_b200", "csrc", "*"))):
+    for f in paths:
         with open(f, "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()
@@ -93,7 +100,7 @@ def ncu_traffic(workload, shapes):
     """Bytes per step for the dominant kernel from the recorded ncu capture, or None if the capture
     does not cover this workload or the kernels have changed since it was taken."""
     table = NCU_TRAFFIC.get(workload)
-    if table is None or kernel_sources_digest() != NCU_TRAFFIC["sources"]:
+    if table is None or kernel_sources_digest(table["sources"]) != table["digest"]:
         return None
     if "per_row_of" in table:
         # one captured shape; the others share its K and N, and traffic grows in proportion to the rows
@@ -102,7 +109,7 @@ def ncu_traffic(workload, shapes):
             return None
         return float(table["bytes"]) * sum(M for (M, K, N) in shapes) / M0
     try:
-        return float(sum(table[tuple(s)] for s in shapes))
+        return float(sum(table["shapes"][tuple(s)] for s in shapes))
     except KeyError:
         return None
 
@@ -494,7 +501,41 @@ def block_sweep(bro, synth, peaks, blocks, groups):
         per_block[str(b if b else K)] = {"us": round(ms * 1e3, 2), "gbs": round(gbs, 1),
                                          "frac_of_measured_copy": round(gbs / peaks["hbm_gbs"], 4),
                                          "frac_of_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4)}
+    # The rotation fused into its producer (Sec. 4.3: the online rotation sits before down_proj, whose
+    # input is silu(gate) * up): one launch that reads gate and up and writes codes and scales (4.53125 B
+    # per element) against the two-step path, producer kernel then rotate+quantize (8.53125 B per element).
+    gates = [(x * 0.5).to(torch.bfloat16) for x in xs]
+    ups = [torch.randn((M, K), dtype=torch.float32, device="cuda", generator=torch.Generator(device="cuda").manual_seed(r)).to(torch.bfloat16)
+           for r in range(ring)]
+    h = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+
+    def fused(i):
+        bro.swiglu_rotate_quantize_mxfp4(gates[i % ring], ups[i % ring], 32, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+
+    def two_step(i):
+        bro.swiglu_bf16(gates[i % ring], ups[i % ring], h)
+        bro.rotate_quantize_mxfp4(h, 32, codes[i % ring], scales[i % ring], bro.LAYOUT_GEMM)
+
+    producer = {}
+    for name, fn, nbytes in (("fused", fused, 4.53125), ("two_step", two_step, 8.53125)):
+        for i in range(3):
+            fn(i)
+        ts = []
+        for gi in range(groups):
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(group):
+                fn(i)
+            c.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(c) / group)
+        ms = statistics.mean(ts)
+        producer[name] = {"us": round(ms * 1e3, 2), "algorithmic_bytes": M * K * nbytes,
+                          "gbs": round(M * K * nbytes / (ms * 1e-3) / 1e9, 1)}
+    producer["speedup"] = round(producer["two_step"]["us"] / producer["fused"]["us"], 3)
+    del gates, ups, h
     return {"shape_MK": [M, K], "algorithmic_bytes": bytes_per_launch, "per_block": per_block,
+            "swiglu_producer_block32": producer,
             "timing": f"CUDA events around groups of {group} back-to-back launches, {groups} groups per size"}, (xs, codes, scales)
 
 

@@ -153,6 +153,33 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
                       int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The rotation fused into its producer.  The one rotation paid at inference sits before down_proj
+ * (Sec. 4.3, "Reduced online computing"; Sec. 6), whose input in the LLaMA-family models the paper
+ * evaluates is the gated activation h = silu(gate) * up.  These entry points compute h inside the
+ * rotate+quantize kernel, so h is never written to or read from device memory:
+ *   h[m, k] = bf16_rne( (g * sigmoid(g)) * u ),  g = gate[m, k], u = up[m, k]  (bf16 in, fp32 arithmetic)
+ * with sigmoid from a fixed sequence of IEEE fp32 operations — e = exp(-|g|) by n = rint(-|g| log2e), two
+ * fused multiply-adds of range reduction, a degree-6 Horner polynomial and an exact scaling by 2^n; e = 0
+ * below -86; sigmoid = (g >= 0 ? 1 : e) / (1 + e) — accurate to a few fp32 ulps and bit-reproducible (the
+ * paper does not spell the producer out; this is the library's reading).  Then the activation path of
+ * bro_rotate_quantize_mxfp4 on h.
+ *   gate_bf16, up_bf16  [M, K] bf16, row strides ldg / ldu in elements (>= K, multiples of 8), 16-byte aligned.
+ *   block               32, 64 or 128 (block = 0 is not offered here: BRO_ERR_UNSUPPORTED).
+ *   signs_bf16          NULL or the +-1 vector of the randomised rotation.
+ * bro_swiglu_bf16 is the producer alone (h as a bf16 tensor [M, ldh]), for callers that need h itself.
+ * bro_swiglu_linear is bro_linear(_rs) with the fused producer in front: y = Q(h R) Q(W R)^T.
+ */
+bro_status bro_swiglu_rotate_quantize_mxfp4(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K,
+                                            int64_t ldg, int64_t ldu, int block, const void* signs_bf16,
+                                            void* codes, void* scales, bro_layout layout, void* stream);
+bro_status bro_swiglu_bf16(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K, int64_t ldg,
+                           int64_t ldu, void* h_bf16, int64_t ldh, void* stream);
+bro_status bro_swiglu_linear(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K, int64_t ldg,
+                             int64_t ldu, int block, const void* signs_bf16, const void* wcodes,
+                             const void* wscales, int64_t N, void* y_bf16, int64_t ldy, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/*
  * Packed weights with a descriptor.  bro_pack_weights writes two bare buffers; nothing in them says
  * which rotation they were packed with, so bro_linear cannot notice weights packed with another block
  * size or sign vector (the rotation would no longer cancel, Eq. 1, and the layer would silently

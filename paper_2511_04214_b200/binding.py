@@ -30,6 +30,7 @@ EXPORTS = [
     "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
     "bro_group_scale_bytes", "bro_outlier_workspace_bytes", "bro_outlier_groups", "bro_scale_histogram",
     "bro_scale_inflation", "bro_pack_weights_desc", "bro_linear_packed",
+    "bro_swiglu_rotate_quantize_mxfp4", "bro_swiglu_bf16", "bro_swiglu_linear",
 ]
 
 
@@ -112,6 +113,12 @@ def _load() -> ctypes.CDLL:
     L.bro_scale_histogram.argtypes = [p, p, i64, p, p]
     L.bro_scale_inflation.restype = ci
     L.bro_scale_inflation.argtypes = [p, p, p, i64, p, p]
+    L.bro_swiglu_rotate_quantize_mxfp4.restype = ci
+    L.bro_swiglu_rotate_quantize_mxfp4.argtypes = [p, p, i64, i64, i64, i64, ci, p, p, p, ci, p]
+    L.bro_swiglu_bf16.restype = ci
+    L.bro_swiglu_bf16.argtypes = [p, p, i64, i64, i64, i64, p, i64, p]
+    L.bro_swiglu_linear.restype = ci
+    L.bro_swiglu_linear.argtypes = [p, p, i64, i64, i64, i64, ci, p, p, p, i64, p, i64, p, sz, p]
     L.bro_pack_weights_desc.restype = ci
     L.bro_pack_weights_desc.argtypes = [p, i64, i64, i64, ci, p, p, p, ctypes.POINTER(PackedWeights), p]
     L.bro_linear_packed.restype = ci
@@ -393,3 +400,32 @@ def linear_packed(x: torch.Tensor, block: int, weights: PackedWeights, y: torch.
     _check(lib.bro_linear_packed(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), ctypes.byref(weights), _ptr(y),
                                  _ld(y, weights.N), _ptr(workspace), workspace.numel(), _stream(stream)),
            "bro_linear_packed")
+
+
+def swiglu_rotate_quantize_mxfp4(gate: torch.Tensor, up: torch.Tensor, block: int, codes, scales,
+                                 layout: int = LAYOUT_GEMM, signs: torch.Tensor = None, stream=None) -> None:
+    """rotate_quantize_mxfp4 of h = silu(gate) * up, with h computed inside the kernel."""
+    assert gate.dtype == up.dtype == torch.bfloat16 and gate.shape == up.shape
+    assert gate.stride(1) == 1 and up.stride(1) == 1
+    M, K = gate.shape
+    _check(lib.bro_swiglu_rotate_quantize_mxfp4(_ptr(gate), _ptr(up), M, K, _ld(gate, K), _ld(up, K), block, _ptr(signs),
+                                                _ptr(codes), _ptr(scales), layout, _stream(stream)),
+           "bro_swiglu_rotate_quantize_mxfp4")
+
+
+def swiglu_bf16(gate: torch.Tensor, up: torch.Tensor, h: torch.Tensor, stream=None) -> None:
+    """h = bf16(silu(gate) * up): the producer alone."""
+    assert gate.dtype == up.dtype == h.dtype == torch.bfloat16 and gate.shape == up.shape == h.shape
+    M, K = gate.shape
+    _check(lib.bro_swiglu_bf16(_ptr(gate), _ptr(up), M, K, _ld(gate, K), _ld(up, K), _ptr(h), _ld(h, K), _stream(stream)),
+           "bro_swiglu_bf16")
+
+
+def swiglu_linear(gate: torch.Tensor, up: torch.Tensor, block: int, wcodes, wscales, N: int, y: torch.Tensor,
+                  workspace: torch.Tensor, signs: torch.Tensor = None, stream=None) -> None:
+    """linear(_rs) on h = silu(gate) * up with the producer fused into rotate+quantize."""
+    assert gate.dtype == up.dtype == y.dtype == torch.bfloat16 and gate.shape == up.shape
+    M, K = gate.shape
+    _check(lib.bro_swiglu_linear(_ptr(gate), _ptr(up), M, K, _ld(gate, K), _ld(up, K), block, _ptr(signs), _ptr(wcodes),
+                                 _ptr(wscales), N, _ptr(y), _ld(y, N), _ptr(workspace), workspace.numel(),
+                                 _stream(stream)), "bro_swiglu_linear")

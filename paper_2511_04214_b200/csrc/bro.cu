@@ -159,10 +159,28 @@ __global__ void expire_wait_kernel(uint64_t budget_ns) {
   bro::mbar_wait(b, 0u, bro::SITE_SELF_TEST, budget_ns);
 }
 
+// h = bf16(silu(gate) * up), 8 values per thread (the producer alone; see rqd::silu_mul).
+__global__ void __launch_bounds__(256) swiglu_kernel(const uint16_t* gate, const uint16_t* up, int64_t M, int64_t K,
+                                                     int64_t ldg, int64_t ldu, uint16_t* h, int64_t ldh) {
+  bro::griddep_wait();
+  bro::griddep_launch_dependents();
+  const int64_t chunks = K >> 3, total = M * chunks;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = i / chunks, c = i - row * chunks;
+    const uint4 g = __ldg(reinterpret_cast<const uint4*>(gate + row * ldg + c * 8));
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(up + row * ldu + c * 8));
+    *reinterpret_cast<uint4*>(h + row * ldh + c * 8) = bro::rqd::swiglu_bf16x8(g, u);
+  }
+}
+
 // ---- rotate + quantise ---------------------------------------------------------------------------
 bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, int block,
                                   const void* signs, void* codes, void* scales, bro_layout layout,
-                                  uint32_t flags, cudaStream_t st) {
+                                  uint32_t flags, cudaStream_t st, const void* up = nullptr, int64_t ldu = 0) {
+  // (up != nullptr: x is the gate of the fused producer, the rotated tensor is silu(x) * up)
+  if (up && (ldu < K || ldu % 8 != 0)) return ldu < K ? BRO_ERR_SHAPE : BRO_ERR_ALIGN;
+  if (up && !aligned(up, 16)) return BRO_ERR_ALIGN;
+  if (up && block == 0) return BRO_ERR_UNSUPPORTED;
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (M == 0 && (layout == BRO_LAYOUT_CANONICAL || layout == BRO_LAYOUT_GEMM)) return BRO_OK;
@@ -191,9 +209,13 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   bool direct = can_direct && (B == 32 || M * K <= ((int64_t)1 << 23));
   if (flags & BRO_FLAG_RQ_TMA_RING) direct = false;
   else if (flags & BRO_FLAG_RQ_DIRECT) direct = can_direct;
+  if (up) {                       // the fused producer exists in the register-streaming kernel only
+    if (!can_direct) return BRO_ERR_UNSUPPORTED;
+    direct = true;
+  }
   if (direct)
     return bro::rqd::launch(x, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs, codes, scales, layout,
-                            gemm_scale_kblocks(K), di.sm_count, st);
+                            gemm_scale_kblocks(K), di.sm_count, st, up, ldu);
 
   CUtensorMap tmx;
   rc = make_map_2d(&tmx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, (uint64_t)K, (uint64_t)M,
@@ -583,6 +605,56 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
   if (!signs_bf16) return BRO_ERR_NULL;
   return linear_impl(x_bf16, M, K, ldx, block, signs_bf16, wcodes, wscales, N, y_bf16, ldy, workspace,
                      workspace_bytes, 0u, stream);
+}
+
+bro_status bro_swiglu_rotate_quantize_mxfp4(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K, int64_t ldg,
+                                            int64_t ldu, int block, const void* signs_bf16, void* codes, void* scales,
+                                            bro_layout layout, void* stream) {
+  if (M > 0 && !up_bf16) return BRO_ERR_NULL;
+  if (block == 0) return BRO_ERR_UNSUPPORTED;
+  return launch_rotate_quantize(gate_bf16, M, K, ldg, block, signs_bf16, codes, scales, layout, 0u,
+                                static_cast<cudaStream_t>(stream), up_bf16, ldu);
+}
+
+bro_status bro_swiglu_bf16(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K, int64_t ldg, int64_t ldu,
+                           void* h_bf16, int64_t ldh, void* stream) {
+  if (M < 0 || K <= 0 || K % 8 != 0 || ldg < K || ldu < K || ldh < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (M == 0) return BRO_OK;
+  if (!gate_bf16 || !up_bf16 || !h_bf16) return BRO_ERR_NULL;
+  if (ldg % 8 != 0 || ldu % 8 != 0 || ldh % 8 != 0 || !aligned(gate_bf16, 16) || !aligned(up_bf16, 16) || !aligned(h_bf16, 16))
+    return BRO_ERR_ALIGN;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  const int64_t want = (M * (K / 8) + 255) / 256, cap = (int64_t)di.sm_count * 8;
+  return bro::cuda_ok(bro::launch_kernel(swiglu_kernel, (unsigned)(want < cap ? want : cap), 256, 0,
+                                         static_cast<cudaStream_t>(stream), 1, static_cast<const uint16_t*>(gate_bf16),
+                                         static_cast<const uint16_t*>(up_bf16), M, K, ldg, ldu,
+                                         static_cast<uint16_t*>(h_bf16), ldh),
+                      "swiglu launch")
+             ? BRO_OK
+             : BRO_ERR_CUDA;
+}
+
+bro_status bro_swiglu_linear(const void* gate_bf16, const void* up_bf16, int64_t M, int64_t K, int64_t ldg, int64_t ldu,
+                             int block, const void* signs_bf16, const void* wcodes, const void* wscales, int64_t N,
+                             void* y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || K % kGroup != 0) return BRO_ERR_SHAPE;
+  if (M == 0 || N == 0) return BRO_OK;
+  if (!gate_bf16 || !up_bf16 || !wcodes || !wscales || !y_bf16 || !workspace) return BRO_ERR_NULL;
+  if (block == 0) return BRO_ERR_UNSUPPORTED;
+  if (!aligned(workspace, 1024)) return BRO_ERR_ALIGN;
+  if (workspace_bytes < bro_linear_workspace_bytes(M, N, K)) return BRO_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint8_t* acodes = ws;
+  uint8_t* ascales = acodes + align_up(bro_codes_bytes(M, K), 1024);
+  uint8_t* gws = ascales + align_up(bro_scales_bytes(M, K, BRO_LAYOUT_GEMM), 1024);
+  bro_status rc = launch_rotate_quantize(gate_bf16, M, K, ldg, block, signs_bf16, acodes, ascales, BRO_LAYOUT_GEMM, 0u,
+                                         static_cast<cudaStream_t>(stream), up_bf16, ldu);
+  if (rc != BRO_OK) return rc;
+  return gemm_impl(acodes, ascales, wcodes, wscales, M, N, K, y_bf16, ldy, BRO_OUT_BF16, gws,
+                   bro_gemm_workspace_bytes(M, N, K), 0u, stream, true);
 }
 
 bro_status bro_pack_weights_desc(const void* w_bf16, int64_t N, int64_t K, int64_t ldw, int block,

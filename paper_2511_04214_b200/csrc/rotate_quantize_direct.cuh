@@ -38,18 +38,60 @@ struct Params {
   int groups_padded;            // groups per row it covers (scale padding included)
   int chunks_per_row;           // ceil(groups_padded / 32)
   int total_tasks;              // rows_padded * chunks_per_row; one task = one warp, 32 groups of a row
+  const uint16_t* up;           // PRODUCER kernels: the second operand of h = silu(x) * up, [M, K] with row stride ldu
+  int64_t ldu;
   float* mse;                   // STATS kernels: [M, K/32] per-group quantisation error instead of codes/scales
   int format;                   // STATS kernels: which 4-bit format (see rq::group_error), or
                                 // rq::kFormatScaleOnly: write the E8M0 byte to scales[M, K/32] and nothing else
 };
+
+// ---- the producer fused in front of the rotation (PRODUCER = 1) ------------------------------------------
+// The online rotation sits before down_proj (paper Sec. 4.3, "Reduced online computing"), whose input in
+// the LLaMA-family models is h = silu(gate) * up.  Computing h inside this kernel saves writing it to HBM
+// and reading it back (4 of 8.5 bytes per element).  The arithmetic is a fixed sequence of IEEE fp32
+// operations (one rounding each), so that it can be reproduced bit for bit elsewhere:
+//   t = -|g|;  n = rint(t log2e);  r = fma(n, -ln2_hi, t);  r = fma(n, -ln2_lo, r);
+//   p = 1 + r (1 + r (1/2 + r (1/6 + r (1/24 + r (1/120 + r/720)))))  (Horner, fma);  e = p 2^n  (0 if t < -86);
+//   h = bf16_rne((g * ((g >= 0 ? 1 : e) / (1 + e))) * u).
+__device__ __forceinline__ float silu_mul(float g, float u) {
+  const float t = -fabsf(g);
+  const float n = rintf(__fmul_rn(t, __uint_as_float(0x3FB8AA3Bu)));
+  float r = __fmaf_rn(n, -__uint_as_float(0x3F317218u), t);
+  r = __fmaf_rn(n, -__uint_as_float(0xB102E308u), r);
+  float p = __uint_as_float(0x3AB60B61u);
+  p = __fmaf_rn(p, r, __uint_as_float(0x3C088889u));
+  p = __fmaf_rn(p, r, __uint_as_float(0x3D2AAAABu));
+  p = __fmaf_rn(p, r, __uint_as_float(0x3E2AAAABu));
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  float e = __uint_as_float(__float_as_uint(p) + ((uint32_t)(int)n << 23));   // p in [0.70, 1.42], n in [-124, 0]: exact
+  e = t >= -86.0f ? e : 0.0f;
+  const float s = __fdiv_rn(g >= 0.0f ? 1.0f : e, __fadd_rn(1.0f, e));
+  return __fmul_rn(__fmul_rn(g, s), u);
+}
+// 8 bf16 gates and 8 bf16 ups -> 8 bf16 values of h
+__device__ __forceinline__ uint4 swiglu_bf16x8(uint4 g, uint4 u) {
+  const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
+  uint32_t h[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float lo = silu_mul(__uint_as_float(gw[k] << 16), __uint_as_float(uw[k] << 16));
+    const float hi = silu_mul(__uint_as_float(gw[k] & 0xFFFF0000u), __uint_as_float(uw[k] & 0xFFFF0000u));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(h[k]) : "f"(hi), "f"(lo));
+  }
+  return make_uint4(h[0], h[1], h[2], h[3]);
+}
 
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
 // (rq::group_error) — the analysis behind the paper's regular-block / outlier-block comparison.
 #ifndef BRO_RQD_WIDE_BLOCKS
 #define BRO_RQD_WIDE_BLOCKS 3
 #endif
-template <int LOG2B, bool SIGNS, bool STATS>
-__global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WIDE_BLOCKS : 3) rotate_quantize_direct_kernel(const Params p) {
+// PRODUCER: the rotated tensor is h = silu(x) * up (see silu_mul), computed here from the two bf16 inputs.
+template <int LOG2B, bool SIGNS, bool STATS, bool PRODUCER = false>
+__global__ void __launch_bounds__(kThreads, PRODUCER ? 2 : ((LOG2B >= 6 && !STATS) ? BRO_RQD_WIDE_BLOCKS : 3))
+rotate_quantize_direct_kernel(const Params p) {
   const int lane = threadIdx.x & 31;
   const int num_warps = (int)gridDim.x * kWarps;
   const int ng = (int)(p.K >> 5);
@@ -68,13 +110,18 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
   constexpr bool kSplit = LOG2B >= 6 && !STATS;
   const int hswz = (kSplit && (lane & 1)) ? 2 : 0;
 
-  auto load = [&](int r, int c, uint4 (&q)[4]) {
+  auto load = [&](int r, int c, uint4 (&q)[4], uint4 (&qu)[4]) {
     const int g = c * 32 + lane;
     if (r < p.M && g < ng) {
       const uint4* src = reinterpret_cast<const uint4*>(p.x + (int64_t)r * p.ldx + (int64_t)g * 32);
 #pragma unroll
       for (int j = 0; j < 4; ++j) q[j] = __ldg(src + (j ^ hswz));
-      if (SIGNS) {
+      if (PRODUCER) {
+        const uint4* usrc = reinterpret_cast<const uint4*>(p.up + (int64_t)r * p.ldu + (int64_t)g * 32);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) qu[j] = __ldg(usrc + (j ^ hswz));
+      }
+      if (SIGNS && !PRODUCER) {
         const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)g * 32);
 #pragma unroll
         for (int j = 0; j < 4; ++j) q[j] = rq::apply_signs(q[j], __ldg(sp + (j ^ hswz)));
@@ -82,17 +129,32 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j) q[j] = make_uint4(0u, 0u, 0u, 0u);   // padding quantises to zeros
+      if (PRODUCER) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) qu[j] = make_uint4(0u, 0u, 0u, 0u);   // (silu(0) * 0 = 0)
+      }
     }
   };
 
-  uint4 cur[4], nxt[4];
-  if (task < p.total_tasks) load(row, chunk, cur);
+  uint4 cur[4], nxt[4], cur_u[4], nxt_u[4];
+  if (task < p.total_tasks) load(row, chunk, cur, cur_u);
   while (task < p.total_tasks) {
     // the next task of this warp: issue its loads now, use them in the next iteration
     const int ntask = task + num_warps;
     int nrow = row + step_row, nchunk = chunk + step_chunk;
     if (nchunk >= p.chunks_per_row) { nchunk -= p.chunks_per_row; ++nrow; }
-    if (ntask < p.total_tasks) load(nrow, nchunk, nxt);
+    if (ntask < p.total_tasks) load(nrow, nchunk, nxt, nxt_u);
+
+    if (PRODUCER) {
+      // h = silu(gate) * up, rounded to bf16: from here on the kernel is the plain one on h
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cur[j] = swiglu_bf16x8(cur[j], cur_u[j]);
+      if (SIGNS && row < p.M && chunk * 32 + lane < ng) {
+        const uint4* sp = reinterpret_cast<const uint4*>(p.signs + (int64_t)(chunk * 32 + lane) * 32);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cur[j] = rq::apply_signs(cur[j], __ldg(sp + (j ^ hswz)));
+      }
+    }
 
     uint64_t P[16];
 #pragma unroll
@@ -137,7 +199,7 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
         }
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+      for (int j = 0; j < 4; ++j) { cur[j] = nxt[j]; if (PRODUCER) cur_u[j] = nxt_u[j]; }
       task = ntask;
       row = nrow;
       chunk = nchunk;
@@ -155,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
         if (live) p.mse[(int64_t)row * ng + g] = e;
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+      for (int j = 0; j < 4; ++j) { cur[j] = nxt[j]; if (PRODUCER) cur_u[j] = nxt_u[j]; }
       task = ntask;
       row = nrow;
       chunk = nchunk;
@@ -184,7 +246,7 @@ __global__ void __launch_bounds__(kThreads, (LOG2B >= 6 && !STATS) ? BRO_RQD_WID
       }
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
+    for (int j = 0; j < 4; ++j) { cur[j] = nxt[j]; if (PRODUCER) cur_u[j] = nxt_u[j]; }
     task = ntask;
     row = nrow;
     chunk = nchunk;
@@ -198,9 +260,9 @@ inline bool supports(int64_t M, int64_t K, bro_layout layout, int64_t scale_kblo
   return rows * ((groups + 31) / 32) < ((int64_t)1 << 30);
 }
 
-template <int LOG2B, bool SIGNS, bool STATS>
+template <int LOG2B, bool SIGNS, bool STATS, bool PRODUCER = false>
 inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
-  auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS, STATS>;
+  auto kernel = rotate_quantize_direct_kernel<LOG2B, SIGNS, STATS, PRODUCER>;
   static DeviceOnce once;            // (one per template instantiation)
   int blocks_per_sm = 1;
   const bro_status rc = device_once(once, &blocks_per_sm, [&](int* n) {
@@ -216,26 +278,30 @@ inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
                                                                                                        : BRO_ERR_CUDA;
 }
 
-template <bool STATS>
+template <bool STATS, bool PRODUCER = false>
 inline bro_status launch_any(Params& p, int log2b, int sm_count, cudaStream_t st) {
   if (p.signs) {
     switch (log2b) {
-      case 5: return launch_one<5, true, STATS>(p, sm_count, st);
-      case 6: return launch_one<6, true, STATS>(p, sm_count, st);
-      default: return launch_one<7, true, STATS>(p, sm_count, st);
+      case 5: return launch_one<5, true, STATS, PRODUCER>(p, sm_count, st);
+      case 6: return launch_one<6, true, STATS, PRODUCER>(p, sm_count, st);
+      default: return launch_one<7, true, STATS, PRODUCER>(p, sm_count, st);
     }
   }
   switch (log2b) {
-    case 5: return launch_one<5, false, STATS>(p, sm_count, st);
-    case 6: return launch_one<6, false, STATS>(p, sm_count, st);
-    default: return launch_one<7, false, STATS>(p, sm_count, st);
+    case 5: return launch_one<5, false, STATS, PRODUCER>(p, sm_count, st);
+    case 6: return launch_one<6, false, STATS, PRODUCER>(p, sm_count, st);
+    default: return launch_one<7, false, STATS, PRODUCER>(p, sm_count, st);
   }
 }
 
+// `up` != nullptr: x is the gate and the rotated tensor is silu(x) * up (the fused producer).
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int log2b, const void* signs, void* codes,
-                         void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+                         void* scales, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st,
+                         const void* up = nullptr, int64_t ldu = 0) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
+  p.up = static_cast<const uint16_t*>(up);
+  p.ldu = ldu;
   p.M = M; p.K = K; p.ldx = ldx;
   p.codes = static_cast<uint8_t*>(codes);
   p.scales = static_cast<uint8_t*>(scales);
@@ -248,7 +314,7 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int l
   p.groups_padded = (int)(layout == BRO_LAYOUT_GEMM ? scale_kblocks * 4 : K / 32);
   p.chunks_per_row = (p.groups_padded + 31) / 32;
   p.total_tasks = p.rows_padded * p.chunks_per_row;
-  return launch_any<false>(p, log2b, sm_count, st);
+  return up ? launch_any<false, true>(p, log2b, sm_count, st) : launch_any<false>(p, log2b, sm_count, st);
 }
 
 // Per-group quantisation error only: mse[M, K/32] (fp32) — or, with format = rq::kFormatScaleOnly, the
@@ -257,6 +323,8 @@ inline bro_status launch_stats(const void* x, int64_t M, int64_t K, int64_t ldx,
                                int format, float* mse, uint8_t* scale_bytes, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
+  p.up = nullptr;
+  p.ldu = 0;
   p.M = M; p.K = K; p.ldx = ldx;
   p.codes = nullptr;
   p.scales = scale_bytes;

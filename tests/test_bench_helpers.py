@@ -10,17 +10,17 @@ import bench  # noqa: E402
 
 def test_traffic_is_null_when_the_kernels_changed(monkeypatch):
     big = [(1024, 8192, 28672), (8192, 8192, 28672), (32768, 8192, 28672)]
-    monkeypatch.setattr(bench, "kernel_sources_digest", lambda: bench.NCU_TRAFFIC["sources"])
     captured = bench.NCU_TRAFFIC["cfg5"]
+    monkeypatch.setattr(bench, "kernel_sources_digest", lambda files=None: captured["digest"])
     assert captured["per_row_of"] == (8192, 8192, 28672)
     # the captured shape itself, and the record over all tensor-bound shapes: scaled by the rows processed
     assert bench.ncu_traffic("cfg5", [(8192, 8192, 28672)]) == float(captured["bytes"])
     assert bench.ncu_traffic("cfg5", big) == float(captured["bytes"]) * (1024 + 8192 + 32768) / 8192
     assert bench.ncu_traffic("cfg5", [(8192, 4096, 28672)]) is None          # another weight matrix: no figure
-    assert bench.ncu_traffic("cfg3", [(4096, 4096, 14336)]) == float(bench.NCU_TRAFFIC["cfg3"][(4096, 4096, 14336)])
+    assert bench.ncu_traffic("cfg3", [(4096, 4096, 14336)]) == float(bench.NCU_TRAFFIC["cfg3"]["shapes"][(4096, 4096, 14336)])
     assert bench.ncu_traffic("cfg3", [(4096, 4096, 4096)]) is None
     assert bench.ncu_traffic("cfg2", [(2048, 2048, 2048)]) is None
-    monkeypatch.setattr(bench, "kernel_sources_digest", lambda: "something else")
+    monkeypatch.setattr(bench, "kernel_sources_digest", lambda files=None: "something else")
     assert bench.ncu_traffic("cfg5", big) is None
 
 
@@ -34,3 +34,5 @@ def test_kernel_label_follows_the_dispatch_rule():
 def test_digest_covers_the_kernel_sources():
     d = bench.kernel_sources_digest()
     assert len(d) == 64 and d == bench.kernel_sources_digest()
+    g = bench.kernel_sources_digest(bench.GEMM_SOURCES)
+    assert g != d and g != bench.kernel_sources_digest(bench.RQ_SOURCES)
