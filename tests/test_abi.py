@@ -121,3 +121,28 @@ def test_packed_weight_descriptor_is_checked_before_any_device_work(lib):
     out = lib.PackedWeights(magic=0x344F5242)
     assert L.bro_pack_weights_desc(p(a), 8, 48, 48, 32, None, p(a), p(a), ctypes.byref(out), None) == 2
     assert out.magic == 0
+
+
+def test_fused_producer_argument_validation_needs_no_device(lib):
+    L = lib.lib
+    buf = (ctypes.c_uint8 * 4096)()
+    a = (ctypes.addressof(buf) + 15) // 16 * 16
+    p = ctypes.c_void_p
+    f = L.bro_swiglu_rotate_quantize_mxfp4
+    assert f(p(a), None, 1, 64, 64, 64, 32, None, p(a), p(a), 0, None) == 1          # up missing
+    assert f(p(a), p(a), 1, 64, 64, 64, 0, None, p(a), p(a), 0, None) == 4           # no full-dimension form
+    assert f(p(a), p(a), 1, 64, 64, 32, 32, None, p(a), p(a), 0, None) == 2          # ldu < K
+    assert f(p(a), p(a), 1, 64, 64, 68, 32, None, p(a), p(a), 0, None) == 3          # ldu not a multiple of 8
+    assert f(p(a), p(a + 2), 1, 64, 64, 64, 32, None, p(a), p(a), 0, None) == 3      # up misaligned
+    assert f(p(a), p(a), 1, 48, 48, 48, 32, None, p(a), p(a), 0, None) == 2          # K not a multiple of 32
+    assert f(p(a), p(a), 0, 64, 64, 64, 32, None, p(a), p(a), 0, None) == 0          # nothing to do
+    g = L.bro_swiglu_bf16
+    assert g(p(a), p(a), 1, 60, 64, 64, p(a), 64, None) == 2                          # K not a multiple of 8
+    assert g(p(a), None, 1, 64, 64, 64, p(a), 64, None) == 1
+    assert g(p(a), p(a), 1, 64, 64, 64, p(a), 32, None) == 2                          # ldh < K
+    assert g(p(a), p(a), 0, 64, 64, 64, p(a), 64, None) == 0
+    a1k = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+    h = L.bro_swiglu_linear
+    assert h(p(a), p(a), 4, 64, 64, 64, 0, None, p(a), p(a), 8, p(a), 8, p(a1k), 1 << 20, None) == 4
+    assert h(p(a), p(a), 4, 64, 64, 64, 32, None, p(a), p(a), 8, p(a), 8, None, 0, None) == 1
+    assert h(p(a), p(a), 4, 64, 64, 64, 32, None, p(a), p(a), 8, p(a), 8, p(a1k), 16, None) == 5
