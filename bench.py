@@ -78,8 +78,8 @@ NCU_TRAFFIC = {
              "per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
     "cfg3": {"sources": GEMM_SOURCES, "digest": "096c61cb1b9865ca985e775b0d340c5efb1060c2d39547c30f96dd9d3d65fab1",
              "shapes": {(4096, 4096, 14336): 68345088 + 69353728}},
-    "cfg4": {"sources": RQ_SOURCES, "digest": "bc16a8ba6dae54c818860574944bc99492436219038af4a402a31e42a0d94714",
-             "shapes": {(16384, 4096, 32): 134230016 + 18973440}},
+    "cfg4": {"sources": RQ_SOURCES, "digest": "91b89ce59cda298187bb3e09db9ca4d2fd34c3e67338b4ca45ad15dcc0ea2d1a",
+             "shapes": {(16384, 4096, 32): 134230784 + 19369472}},
 }
 
 

@@ -85,12 +85,9 @@ __device__ __forceinline__ uint4 swiglu_bf16x8(uint4 g, uint4 u) {
 
 // STATS: nothing is quantised to memory; the kernel writes the per-group quantisation error
 // (rq::group_error) — the analysis behind the paper's regular-block / outlier-block comparison.
-#ifndef BRO_RQD_WIDE_BLOCKS
-#define BRO_RQD_WIDE_BLOCKS 3
-#endif
 // PRODUCER: the rotated tensor is h = silu(x) * up (see silu_mul), computed here from the two bf16 inputs.
 template <int LOG2B, bool SIGNS, bool STATS, bool PRODUCER = false>
-__global__ void __launch_bounds__(kThreads, PRODUCER ? 2 : ((LOG2B >= 6 && !STATS) ? BRO_RQD_WIDE_BLOCKS : 3))
+__global__ void __launch_bounds__(kThreads, PRODUCER ? 2 : 3)
 rotate_quantize_direct_kernel(const Params p) {
   const int lane = threadIdx.x & 31;
   const int num_warps = (int)gridDim.x * kWarps;
