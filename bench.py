@@ -11,8 +11,9 @@ M in {1, 16, 128, 1024, 8192, 32768} tokens (the largest single-GPU workload of 
 Prints ONE JSON line (rank 0).  `value` is device-timed throughput with inputs resident in HBM;
 `e2e` is the same metric through the host-buffer entry point (H2D of x and D2H of y inside the
 timed region); `roofline` describes the dominant kernel (the GEMM on the tensor-bound shapes,
-M >= 1024) timed per launch with CUDA events, `decode` the weight-streaming shapes (M <= 128)
-against the HBM copy bandwidth; `per_config` repeats the per-kernel figures for the other
+M >= 1024) timed per launch with CUDA events — its `operand_data_effect` times one of those launches
+on the real operands and on all-zero codes, which separates the kernel from the chip's power
+management —, `decode` the weight-streaming shapes (M <= 128) against the HBM copy bandwidth; `per_config` repeats the per-kernel figures for the other
 workloads (cfg2, cfg3 and the block-size sweep cfg4) in the same process; `cpu_baseline` is the
 CPU oracle on a bounded sample.  With --gpus N > 1 every rank runs an independent replica — the
 path has no cross-GPU exchange; when no launcher has set WORLD_SIZE the script starts its N ranks
