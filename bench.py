@@ -655,7 +655,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             return None
 
-    if world == 1 and not args.randomised:
+    if world == 1 and not args.randomised and not args.no_operand_effect:
         tensor_bound = [i for i, sh in enumerate(shapes) if list(sh) in roofline["shapes"]]
         mid = [i for i in tensor_bound if shapes[i][0] <= 8192] or tensor_bound
         pick = max(mid, key=lambda i: shapes[i][0] * shapes[i][1] * shapes[i][2])
@@ -991,6 +991,8 @@ def main():
                     help="use the randomised block rotation diag(s) H / sqrt(block) (the *_rs entry points)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-operand-effect", action="store_true",
+                    help="skip the zero-codes / real-operands comparison of one GEMM launch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
                     help="skip the per-kernel figures of the other workloads (cfg2, cfg3, cfg4)")
