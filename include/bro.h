@@ -258,6 +258,27 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
                                      void* stream);
 
 /*
+ * Simulated ("fake") quantisation: rotate, quantise, dequantise.  The paper evaluates every method by
+ * simulating the MX formats rather than running a native FP4 GEMM (Sec. 3.1, experimental setup), and
+ * its format study compares MXFP4 with BFP4, MXINT4 and BINT4 on the same tensors (Sec. 3.2 / Fig. 2,
+ * Sec. 4.1 / Fig. 3); this call produces those tensors.  For every row of x:
+ *   deq[m, :] = dequantised values of Q_format((x diag(s) R_block)[m, :]),  fp32, in the ROTATED domain
+ * with the quantisers listed above (decisions as in bro_group_quant_error_fmt).  Every value is a 3-bit
+ * element times a power of two or an fp16 scale, hence exact in fp32; a negative input that quantises
+ * to zero gives -0.0, a group whose fp16 scale rounds to zero gives +0.0 throughout.
+ *   block       1 (no rotation), 32, 64, 128 or 0 (= K, K a power of two in [32, 32768])
+ *   signs_bf16  NULL or the +-1 vector of the randomised rotation (device, [K] bf16, 16-byte aligned)
+ *   deq         device, fp32 [M, K] with row stride ldd >= K elements (ldd % 4 == 0, 16-byte aligned);
+ *               columns K .. ldd-1 are not written
+ * Errors as for bro_group_quant_error_fmt; M == 0 returns BRO_OK without a launch.  Only MXFP4 has a
+ * GEMM in this library: a simulated W4A4 layer in another format is deq_a deq_w^T in the caller's
+ * precision.
+ */
+bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                    const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
+                                    void* stream);
+
+/*
  * Scale statistics behind the paper's regular-block / outlier-block argument (Sec. 4.1: "regular
  * blocks" hold no outlier, "outlier blocks" one or more; Sec. 4.2, Fig. 6 caption: outliers are the
  * top 0.1 % of the activations by absolute value; App. A.3, Fig. 8-9: under global rotation the scales

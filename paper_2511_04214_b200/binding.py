@@ -25,7 +25,7 @@ EXPORTS = [
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host", "bro_linear_static",
-    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt",
+    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt", "bro_rotate_fake_quantize",
     "bro_last_device_status_ex", "bro_selftest_expire_wait",
     "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
     "bro_group_scale_bytes", "bro_outlier_workspace_bytes", "bro_outlier_groups", "bro_scale_histogram",
@@ -101,6 +101,8 @@ def _load() -> ctypes.CDLL:
     L.bro_group_quant_error.argtypes = [p, i64, i64, i64, ci, p, p, p]
     L.bro_group_quant_error_fmt.restype = ci
     L.bro_group_quant_error_fmt.argtypes = [p, i64, i64, i64, ci, p, ci, p, p]
+    L.bro_rotate_fake_quantize.restype = ci
+    L.bro_rotate_fake_quantize.argtypes = [p, i64, i64, i64, ci, p, ci, p, i64, p]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
     L.bro_group_scale_bytes.restype = ci
@@ -337,6 +339,17 @@ def group_quant_error(x: torch.Tensor, block: int, mse: torch.Tensor, signs: tor
     assert mse.shape == (M, K // 32)
     _check(lib.bro_group_quant_error_fmt(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(mse),
                                          _stream(stream)), "bro_group_quant_error_fmt")
+
+
+def rotate_fake_quantize(x: torch.Tensor, block: int, deq: torch.Tensor, fmt: str = "mxfp4", signs: torch.Tensor = None,
+                         stream=None) -> None:
+    """Simulated quantisation: ``deq`` (fp32 [M, K], rows may be strided) receives the dequantised values of
+    x R_block quantised to ``fmt``; block = 1: no rotation, 0: the full dimension."""
+    assert x.dtype == torch.bfloat16 and deq.dtype == torch.float32
+    M, K = x.shape
+    assert deq.shape == (M, K)
+    _check(lib.bro_rotate_fake_quantize(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(deq), _ld(deq, K),
+                                        _stream(stream)), "bro_rotate_fake_quantize")
 
 
 def group_scale_bytes(x: torch.Tensor, block: int, scales: torch.Tensor, signs: torch.Tensor = None, stream=None) -> None:

@@ -13,6 +13,7 @@
 #include "gemm_mxfp4.cuh"
 #include "gemm_mxfp4_2cta.cuh"
 #include "scale_stats.cuh"
+#include "fake_quantize.cuh"
 
 namespace {
 
@@ -378,6 +379,31 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, (int)format, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
   if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
   return bro::rqd::launch_stats(x_bf16, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs_bf16, (int)format, mse, nullptr, di.sm_count, st);
+}
+
+// ---- simulated quantisation ----------------------------------------------------------------------
+bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                    const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
+                                    void* stream) {
+  if ((int)format < 0 || (int)format > 3) return BRO_ERR_SHAPE;
+  if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K || ldd < K) return BRO_ERR_SHAPE;
+  if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
+  if (block != 0 && block != 1 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  const int64_t B = block == 0 ? K : block;
+  if (K % B != 0) return BRO_ERR_SHAPE;
+  if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
+  if (M == 0) return BRO_OK;
+  if (!x_bf16 || !deq) return BRO_ERR_NULL;
+  if (ldx % 8 != 0 || ldd % 4 != 0 || !aligned(x_bf16, 16) || !aligned(deq, 16) || !aligned(signs_bf16, 16))
+    return BRO_ERR_ALIGN;
+  DeviceInfo di;
+  bro_status rc = device_info(&di);
+  if (rc != BRO_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (B > 128)
+    return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, nullptr, (int)format, BRO_LAYOUT_CANONICAL, 0,
+                            di.sm_count, st, deq, ldd);
+  return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, deq, ldd, di.sm_count, st);
 }
 
 // ---- scale statistics ----------------------------------------------------------------------------

@@ -12,6 +12,7 @@
 
 #include "bro_common.cuh"
 #include "rotate_quantize.cuh"
+#include "fake_quantize.cuh"
 
 namespace bro {
 namespace rqg {
@@ -29,6 +30,8 @@ struct Params {
   const uint16_t* signs; // [K] bf16 +-1 for the randomised rotation diag(s) H / sqrt(K), or nullptr
   float* mse;            // if set: write the per-group quantisation error [M, K/32] instead of codes/scales
   int format;            // ... for this 4-bit format (see rq::group_error)
+  float* deq;            // if set: write the dequantised values [M, K] (row stride ldd) under `format` instead
+  int64_t ldd;
 };
 
 template <int kMaxThreads>
@@ -102,6 +105,12 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
     if (p.mse) {                 // analysis mode (uniform over the grid)
       const float e = rq::group_error(P, cbits, p.format);
       if (live) p.mse[row * (p.K >> 5) + gi] = e;
+      continue;
+    }
+    if (p.deq) {                 // simulated quantisation (uniform over the grid)
+      float out[32];
+      fq::group_dequant(P, cbits, p.format, out);
+      if (live) fq::store_group(p.deq + row * p.ldd + (int64_t)gi * 32, out);
       continue;
     }
     uint32_t w[4];
@@ -337,8 +346,11 @@ __global__ void __launch_bounds__(128, 5) rotate_quantize_global_smem_kernel(con
 bro_status make_row_map(CUtensorMap* map, const void* x, int64_t M, int64_t K, int64_t ldx, int box_rows);
 
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
-                         void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st) {
+                         void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st,
+                         float* deq = nullptr, int64_t ldd = 0) {
   Params p;
+  p.deq = deq;
+  p.ldd = ldd;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M;
   p.K = K;
@@ -357,12 +369,12 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   int threads = p.threads_per_row < 256 ? 256 : p.threads_per_row;
   p.rows_per_iter = threads / p.threads_per_row;
   const size_t smem = K > 1024 ? (size_t)p.rows_per_iter * K * sizeof(float) : 0;
-  if (layout == BRO_LAYOUT_GEMM && !mse && format != rq::kFormatScaleOnly) {
+  if (layout == BRO_LAYOUT_GEMM && !mse && !deq && format != rq::kFormatScaleOnly) {
     // padding rows / groups of the tiled scale buffer must read as 0
     const size_t bytes = (size_t)((M + 127) / 128) * (size_t)scale_kblocks * 512;
     if (cudaMemsetAsync(scales, 0, bytes, st) != cudaSuccess) return BRO_ERR_CUDA;
   }
-  if ((K == 2048 || K == 4096) && !mse && format != rq::kFormatScaleOnly) {
+  if ((K == 2048 || K == 4096) && !mse && !deq && format != rq::kFormatScaleOnly) {
     // codes path at these sizes: all stages in registers, two shared-memory transposes
     const int rows = (int)(128 / (K / 32));
     const int64_t iters2 = (M + rows - 1) / rows;

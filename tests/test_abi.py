@@ -95,6 +95,26 @@ def test_argument_validation_needs_no_device(lib):
     assert L.bro_linear(p(a128), 4, 32, 32, 32, p(a128), p(a128), 8, p(a128), 8, None, 0, None) == 1
 
 
+def test_fake_quantize_argument_validation_needs_no_device(lib):
+    L = lib.lib
+    buf = (ctypes.c_uint8 * 4096)()
+    a16 = (ctypes.addressof(buf) + 15) // 16 * 16
+    p = ctypes.c_void_p
+    fq = L.bro_rotate_fake_quantize
+    assert fq(None, 1, 64, 64, 32, None, 0, p(a16), 64, None) == 1
+    assert fq(p(a16), 1, 64, 64, 32, None, 0, None, 64, None) == 1
+    assert fq(p(a16), 1, 64, 64, 32, None, 4, p(a16), 64, None) == 2         # no such format
+    assert fq(p(a16), 1, 48, 48, 32, None, 0, p(a16), 48, None) == 2         # K not a multiple of 32
+    assert fq(p(a16), 1, 64, 64, 16, None, 0, p(a16), 64, None) == 2         # no such block
+    assert fq(p(a16), 1, 96, 96, 64, None, 0, p(a16), 96, None) == 2         # K not a multiple of the block
+    assert fq(p(a16), 1, 64, 64, 32, None, 0, p(a16), 60, None) == 2         # ldd < K
+    assert fq(p(a16), 1, 96, 96, 0, None, 0, p(a16), 96, None) == 4          # full-dimension rotation needs a power of two
+    assert fq(p(a16), 1, 64, 64, 32, None, 0, p(a16), 66, None) == 3         # ldd not a multiple of 4
+    assert fq(p(a16), 1, 64, 64, 32, None, 0, p(a16 + 4), 64, None) == 3
+    assert fq(p(a16), 1, 64, 64, 32, p(a16 + 2), 0, p(a16), 64, None) == 3
+    assert fq(p(a16), 0, 64, 64, 1, None, 3, p(a16), 64, None) == 0          # no rows: nothing to do
+
+
 def test_packed_weight_descriptor_is_checked_before_any_device_work(lib):
     """bro_linear_packed refuses weights packed with another block size, another K, with / without a sign
     vector, or a descriptor that is not one — all on the host, before any CUDA call."""
