@@ -79,8 +79,8 @@ NCU_TRAFFIC = {
              "per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
     "cfg3": {"sources": GEMM_SOURCES, "digest": "096c61cb1b9865ca985e775b0d340c5efb1060c2d39547c30f96dd9d3d65fab1",
              "shapes": {(4096, 4096, 14336): 68345088 + 69353728}},
-    "cfg4": {"sources": RQ_SOURCES, "digest": "91b89ce59cda298187bb3e09db9ca4d2fd34c3e67338b4ca45ad15dcc0ea2d1a",
-             "shapes": {(16384, 4096, 32): 134230784 + 19369472}},
+    "cfg4": {"sources": RQ_SOURCES, "digest": "c4a4fce939241ee08e3b2f6df39852f3df19e86dc45da160525da500e9300102",
+             "shapes": {(16384, 4096, 32): 134231296 + 19468288}},
 }
 
 
@@ -944,6 +944,15 @@ def run_rotate_quantize_only(args):
             bro.group_quant_error(xs[0], b, mse_buf, fmt=fmt)
             format_study[fmt][str(b if b else K)] = {"all": float(mse_buf.mean()), "regular": float(mse_buf[~outlier_gpu].mean()),
                                                      "outlier": float(mse_buf[outlier_gpu].mean())}
+    # Rotation-dimension sweep (Sec. 5.2 / Fig. 7, in error terms): no rotation, the dimensions below the
+    # MX group, the group itself, and above it, MXFP4, same tensor.
+    dimension_sweep = {}
+    if not args.only_block:
+        for b in (1, 2, 4, 8, 16, 32, 64, 128, 0):
+            bro.group_quant_error(xs[0], b, mse_buf)
+            dimension_sweep[str(b if b else K)] = {"all": float(mse_buf.mean()), "regular": float(mse_buf[~outlier_gpu].mean()),
+                                                   "outlier": float(mse_buf[outlier_gpu].mean()),
+                                                   "median": float(mse_buf.flatten()[::7].median())}
     assert bro.last_device_status() == 0
     ms_total = t_all0.elapsed_time(t_all1)
     value = bytes_per_launch * len(blocks) * steps / (ms_total * 1e-3) / 1e9
@@ -955,6 +964,7 @@ def run_rotate_quantize_only(args):
                       "l2": f"ring of {ring} inputs (3 x 134 MB) > 126 MB L2", "layout": "gemm", "flags": args.flags},
            "clocks": sampler.stop(), "gpu_launches": steps * len(blocks), "per_block": per_block,
            "oracle_group_mse": oracle_mse, "gpu_group_mse": gpu_mse, "gpu_format_study": format_study,
+           "gpu_rotation_dimension_sweep": dimension_sweep,
            "roofline": {"bound": "hbm", "kernel": "rotate_quantize_kernel", "achieved": first["gbs"], "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "frac": first["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                         "traffic": ncu_traffic("cfg4", [(M, K, blocks[0] if blocks[0] else K)]),

@@ -234,8 +234,10 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
  * row of x and every group of 32 channels of y = x R_block:
  *   mse[m, g] = mean_i (y_i - deq(Q(y))_i)^2
  * with Q the MXFP4 quantiser of bro_rotate_quantize_mxfp4.  Nothing else is written.
- *   block       32, 64, 128 or 0 (= K), as above;  signs_bf16  NULL or the +-1 vector of the
- *               randomised rotation;  mse  device, fp32 [M, K/32], dense.
+ *   block       32, 64, 128 or 0 (= K), as above; also 1 (no rotation) and 2, 4, 8, 16 (a rotation
+ *               inside the MX group: Sec. 5.2 sweeps the rotation dimension below as well as above
+ *               the group size; these sizes exist in the analysis calls only);
+ *   signs_bf16  NULL or the +-1 vector of the randomised rotation;  mse  device, fp32 [M, K/32], dense.
  * Arithmetic: differences are exact, squares and their sum are rounded in fp32 (relative error of a
  * few 2^-24 against an fp64 evaluation).
  */
@@ -266,7 +268,8 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
  * with the quantisers listed above (decisions as in bro_group_quant_error_fmt).  Every value is a 3-bit
  * element times a power of two or an fp16 scale, hence exact in fp32; a negative input that quantises
  * to zero gives -0.0, a group whose fp16 scale rounds to zero gives +0.0 throughout.
- *   block       1 (no rotation), 32, 64, 128 or 0 (= K, K a power of two in [32, 32768])
+ *   block       1 (no rotation), 2, 4, 8, 16 (inside the MX group), 32, 64, 128 or 0 (= K, K a power
+ *               of two in [32, 32768])
  *   signs_bf16  NULL or the +-1 vector of the randomised rotation (device, [K] bf16, 16-byte aligned)
  *   deq         device, fp32 [M, K] with row stride ldd >= K elements (ldd % 4 == 0, 16-byte aligned);
  *               columns K .. ldd-1 are not written
@@ -287,7 +290,8 @@ bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, in
  *
  * bro_group_scale_bytes: scales[m, g] (uint8 [M, K/32], dense) = the scale byte of group g of row m of
  *   x R_block.  block = 1 is the identity rotation — the activations as they are ("before rotation");
- *   32, 64, 128 and 0 (= K) as in bro_rotate_quantize_mxfp4; signs_bf16 NULL or the +-1 vector.
+ *   2, 4, 8, 16 rotate inside the MX group; 32, 64, 128 and 0 (= K) as in bro_rotate_quantize_mxfp4;
+ *   signs_bf16 NULL or the +-1 vector.
  *   Nothing else is written.
  */
 bro_status bro_group_scale_bytes(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,

@@ -359,6 +359,12 @@ bro_status bro_rotate_quantize_mxfp4_rs(const void* x_bf16, int64_t M, int64_t K
                                 static_cast<cudaStream_t>(stream));
 }
 
+// Rotation sizes of the analysis calls: 0 (= K), 1 (none), and the powers of two from 2 to 128 — below,
+// at and above the MX group (Sec. 5.2 sweeps the rotation dimension both ways).
+static bool analysis_block(int block) {
+  return block == 0 || (block >= 1 && block <= 128 && (block & (block - 1)) == 0);
+}
+
 bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                      const void* signs_bf16, bro_format format, float* mse, void* stream) {
   if ((int)format < 0 || (int)format > 3) return BRO_ERR_SHAPE;
@@ -367,7 +373,7 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
   if (M == 0) return BRO_OK;
   if (!x_bf16 || !mse) return BRO_ERR_NULL;
   const int64_t B = block == 0 ? K : block;
-  if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  if (!analysis_block(block)) return BRO_ERR_SHAPE;
   if (K % B != 0) return BRO_ERR_SHAPE;
   if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
   if (ldx % 8 != 0 || !aligned(x_bf16, 16) || !aligned(mse, 4) || !aligned(signs_bf16, 16)) return BRO_ERR_ALIGN;
@@ -375,6 +381,8 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (B < 32)   // no rotation, or one inside the MX group
+    return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, nullptr, 0, mse, nullptr, di.sm_count, st);
   if (B > 128)
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, mse, (int)format, BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);
   if (!bro::rqd::supports(M, K, BRO_LAYOUT_CANONICAL, 0)) return BRO_ERR_UNSUPPORTED;
@@ -388,7 +396,7 @@ bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, in
   if ((int)format < 0 || (int)format > 3) return BRO_ERR_SHAPE;
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K || ldd < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
-  if (block != 0 && block != 1 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  if (!analysis_block(block)) return BRO_ERR_SHAPE;
   const int64_t B = block == 0 ? K : block;
   if (K % B != 0) return BRO_ERR_SHAPE;
   if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
@@ -403,7 +411,7 @@ bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, in
   if (B > 128)
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, nullptr, (int)format, BRO_LAYOUT_CANONICAL, 0,
                             di.sm_count, st, deq, ldd);
-  return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, deq, ldd, di.sm_count, st);
+  return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, deq, ldd, nullptr, nullptr, di.sm_count, st);
 }
 
 // ---- scale statistics ----------------------------------------------------------------------------
@@ -411,7 +419,7 @@ bro_status bro_group_scale_bytes(const void* x_bf16, int64_t M, int64_t K, int64
                                  const void* signs_bf16, uint8_t* scales, void* stream) {
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
-  if (block != 0 && block != 1 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  if (!analysis_block(block)) return BRO_ERR_SHAPE;
   const int64_t B = block == 0 ? K : block;
   if (K % B != 0) return BRO_ERR_SHAPE;
   if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
@@ -431,6 +439,8 @@ bro_status bro_group_scale_bytes(const void* x_bf16, int64_t M, int64_t K, int64
                ? BRO_OK
                : BRO_ERR_CUDA;
   }
+  if (B < 32)   // a rotation inside the MX group
+    return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, 0, nullptr, 0, nullptr, scales, di.sm_count, st);
   if (B > 128)
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, scales, nullptr, bro::rq::kFormatScaleOnly,
                             BRO_LAYOUT_CANONICAL, 0, di.sm_count, st);

@@ -7,7 +7,9 @@
 // One thread owns one MX group of 32 channels (64 bytes of bf16), a warp 32 consecutive groups of a
 // row; the rotation is the same fixed-order fp32 butterfly as in the quantising kernels (stages of
 // stride 1..16 in registers, stride 32 / 64 through one / two shuffles for blocks of 64 / 128), or
-// none at all (LOG2B = 0: the identity, "before rotation").  Every dequantised value is exactly
+// none at all (LOG2B = 0: the identity, "before rotation"), or a rotation inside the MX group
+// (LOG2B = 1..4: blocks of 2..16 channels — the paper's Sec. 5.2 sweeps the rotation dimension below as
+// well as above the MX group), which simply stops the butterfly early.  Every dequantised value is exactly
 // representable in fp32 (a 3-bit element times a power of two or an 11-bit fp16 scale), so the result
 // can be compared bit for bit with an evaluation in higher precision.
 //
@@ -104,14 +106,32 @@ struct Params {
   const uint16_t* x;
   int64_t M, K, ldx;
   const uint16_t* signs;        // [K] bf16 +-1 (kernels with SIGNS) or nullptr
-  float* deq;                   // [M, K] fp32, row stride ldd
+  float* deq;                   // [M, K] fp32, row stride ldd — or nullptr, and then one of:
   int64_t ldd;
+  float* mse;                   //   [M, K/32] per-group quantisation error (rq::group_error)
+  uint8_t* scale_bytes;         //   [M, K/32] E8M0 byte of each group (rq::group_scale_byte)
   int format;
   int chunks_per_row;           // ceil((K / 32) / 32): one task = one warp, 32 groups of a row
   int64_t total_tasks;          // M * chunks_per_row
 };
 
-// LOG2B = 0: no rotation; 5, 6, 7: blocks of 32, 64, 128.
+// Butterfly stages of stride 2 .. B/2 on pairs, for B <= 16 (pair k meets pair k ^ (h/2)).
+template <int LOG2B>
+__device__ __forceinline__ void fwht_small(uint64_t (&P)[16]) {
+#pragma unroll
+  for (int hp = 1; hp < (1 << (LOG2B - 1)); hp <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if ((k & hp) == 0) {
+        const uint64_t a = P[k], b = P[k + hp];
+        P[k] = rq::add2(a, b);
+        P[k + hp] = rq::sub2(a, b);
+      }
+    }
+  }
+}
+
+// LOG2B = 0: no rotation; 1..4: blocks of 2..16 inside the group; 5, 6, 7: blocks of 32, 64, 128.
 template <int LOG2B, bool SIGNS>
 __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params p) {
   __shared__ __align__(16) float sbuf[kWarps][32 * 32];      // 4 KiB per warp
@@ -119,6 +139,7 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
   float* wbuf = sbuf[threadIdx.x >> 5];
   const int ng = (int)(p.K >> 5);
   constexpr uint32_t cbits = LOG2B == 0 ? 0x3F800000u : rq::norm_bits<(LOG2B == 0 ? 5 : LOG2B)>();
+  const bool full = p.deq != nullptr;             // (uniform over the grid)
   griddep_wait();
   griddep_launch_dependents();
   const int64_t num_warps = (int64_t)gridDim.x * kWarps;
@@ -141,9 +162,20 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
         rq::unpack_stage1(q, P + 4 * j);
       }
     }
-    if (LOG2B != 0) rq::fwht32_stages_2_to_16(P);
+    if (LOG2B >= 5) rq::fwht32_stages_2_to_16(P);
+    if (LOG2B >= 2 && LOG2B <= 4) fwht_small<(LOG2B >= 2 && LOG2B <= 4) ? LOG2B : 2>(P);
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
+    if (!full) {                                   // the statistics only
+      if (p.mse) {
+        const float e = rq::group_error(P, cbits, p.format);
+        if (live) p.mse[row * ng + g] = e;
+      } else {
+        const uint32_t sb = rq::group_scale_byte(P, cbits);
+        if (live) p.scale_bytes[row * ng + g] = (uint8_t)sb;
+      }
+      continue;
+    }
     float out[32];
     group_dequant(P, cbits, p.format, out);
     // lane l -> buffer row l (128 bytes), piece j at position j ^ (l & 7)
@@ -165,14 +197,17 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
   }
 }
 
+// block: 1 (identity), 2, 4, 8, 16, 32, 64 or 128.  Exactly one of deq / mse / scale_bytes is set.
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int block, const void* signs, int format,
-                         float* deq, int64_t ldd, int sm_count, cudaStream_t st) {
+                         float* deq, int64_t ldd, float* mse, uint8_t* scale_bytes, int sm_count, cudaStream_t st) {
   Params p;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M; p.K = K; p.ldx = ldx;
   p.signs = static_cast<const uint16_t*>(signs);
   p.deq = deq;
   p.ldd = ldd;
+  p.mse = mse;
+  p.scale_bytes = scale_bytes;
   p.format = format;
   p.chunks_per_row = (int)((K / 32 + 31) / 32);
   p.total_tasks = M * p.chunks_per_row;
@@ -182,20 +217,29 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int b
   auto go = [&](auto kernel) -> bro_status {
     return cuda_ok(launch_kernel(kernel, grid, kThreads, 0, st, 1, p), "fake_quantize launch") ? BRO_OK : BRO_ERR_CUDA;
   };
-  // (a sign flip commutes with a symmetric quantiser, but it changes which values meet in a butterfly:
-  // with the identity the signs only flip the output signs, and are applied all the same)
+  int lg = 0;
+  while ((1 << lg) < block) ++lg;
+  // (with the identity the signs only flip the output signs; they are applied all the same)
   if (signs) {
-    switch (block) {
-      case 1: return go(fake_quantize_kernel<0, true>);
-      case 32: return go(fake_quantize_kernel<5, true>);
-      case 64: return go(fake_quantize_kernel<6, true>);
+    switch (lg) {
+      case 0: return go(fake_quantize_kernel<0, true>);
+      case 1: return go(fake_quantize_kernel<1, true>);
+      case 2: return go(fake_quantize_kernel<2, true>);
+      case 3: return go(fake_quantize_kernel<3, true>);
+      case 4: return go(fake_quantize_kernel<4, true>);
+      case 5: return go(fake_quantize_kernel<5, true>);
+      case 6: return go(fake_quantize_kernel<6, true>);
       default: return go(fake_quantize_kernel<7, true>);
     }
   }
-  switch (block) {
-    case 1: return go(fake_quantize_kernel<0, false>);
-    case 32: return go(fake_quantize_kernel<5, false>);
-    case 64: return go(fake_quantize_kernel<6, false>);
+  switch (lg) {
+    case 0: return go(fake_quantize_kernel<0, false>);
+    case 1: return go(fake_quantize_kernel<1, false>);
+    case 2: return go(fake_quantize_kernel<2, false>);
+    case 3: return go(fake_quantize_kernel<3, false>);
+    case 4: return go(fake_quantize_kernel<4, false>);
+    case 5: return go(fake_quantize_kernel<5, false>);
+    case 6: return go(fake_quantize_kernel<6, false>);
     default: return go(fake_quantize_kernel<7, false>);
   }
 }

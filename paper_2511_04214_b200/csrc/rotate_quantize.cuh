@@ -376,7 +376,7 @@ __device__ __forceinline__ float group_error(const uint64_t (&P)[16], uint32_t c
   float acc = 0.f;
   if (format == 0 || format == 2) {
     const uint32_t s = format == 0 ? (ef > 2u ? ef - 2u : 0u) : ef;
-    const float inv = __uint_as_float((254u - s) << 23);                    // 2^-E, E = s - 127
+    const float inv = __uint_as_float(s <= 253u ? ((254u - s) << 23) : 0x00400000u);   // 2^-E, E = s - 127 (2^-127 is subnormal)
     const float pe = __uint_as_float(s >= 1u ? (s << 23) : 0x00400000u);    // 2^E (2^-127 is subnormal)
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {

@@ -105,7 +105,8 @@ def test_fake_quantize_argument_validation_needs_no_device(lib):
     assert fq(p(a16), 1, 64, 64, 32, None, 0, None, 64, None) == 1
     assert fq(p(a16), 1, 64, 64, 32, None, 4, p(a16), 64, None) == 2         # no such format
     assert fq(p(a16), 1, 48, 48, 32, None, 0, p(a16), 48, None) == 2         # K not a multiple of 32
-    assert fq(p(a16), 1, 64, 64, 16, None, 0, p(a16), 64, None) == 2         # no such block
+    assert fq(p(a16), 1, 96, 96, 24, None, 0, p(a16), 96, None) == 2         # no such block
+    assert fq(p(a16), 1, 256, 256, 256, None, 0, p(a16), 256, None) == 2
     assert fq(p(a16), 1, 96, 96, 64, None, 0, p(a16), 96, None) == 2         # K not a multiple of the block
     assert fq(p(a16), 1, 64, 64, 32, None, 0, p(a16), 60, None) == 2         # ldd < K
     assert fq(p(a16), 1, 96, 96, 0, None, 0, p(a16), 96, None) == 4          # full-dimension rotation needs a power of two

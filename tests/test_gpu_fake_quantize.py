@@ -48,14 +48,15 @@ def check(got, ref):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("block,M,K", [(1, 37, 416), (32, 37, 416), (64, 37, 448), (128, 37, 640), (32, 300, 4096),
-                                       (0, 37, 512), (0, 21, 2048), (128, 130, 1024)])
+                                       (0, 37, 512), (0, 21, 2048), (128, 130, 1024),
+                                       (2, 37, 416), (4, 37, 416), (8, 37, 416), (16, 37, 416)])
 def test_matches_the_oracle_exactly(bro, fmt, block, M, K):
     x = synth.activations(M, K, seed=300 + M + block)
     check(gpu(bro, x, block, fmt), oracle.fake_quantize(rotated(x, block), fmt))
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
-@pytest.mark.parametrize("block,K", [(1, 416), (32, 416), (128, 640), (0, 1024)])
+@pytest.mark.parametrize("block,K", [(1, 416), (4, 416), (16, 416), (32, 416), (128, 640), (0, 1024)])
 def test_randomised_rotation(bro, fmt, block, K):
     x = synth.activations(45, K, seed=9)
     signs = synth.rotation_signs(K, seed=10)

@@ -112,3 +112,39 @@ def test_randomised_rotation_every_block_size(bro, block, M, K):
     x = synth.activations(M, K, seed=7 + M)
     signs = synth.rotation_signs(K, seed=K + 1)
     check(gpu(bro, x, block, signs), reference(x, block, signs))
+
+
+@pytest.mark.parametrize("fmt", ["mxfp4", "bfp4", "mxint4", "bint4"])
+@pytest.mark.parametrize("block", [1, 2, 4, 8, 16])
+def test_rotations_inside_the_mx_group(bro, fmt, block):
+    """No rotation and the rotation dimensions below the MX group (Sec. 5.2 sweeps the dimension both
+    ways), with and without random signs; block 1 is compared with the oracle on the plain activations."""
+    M, K = 67, 416
+    x = synth.activations(M, K, seed=500 + block)
+    signs = synth.rotation_signs(K, seed=501)
+    for sg in (None, signs):
+        if block == 1:
+            y = x.float().numpy() * (1.0 if sg is None else sg.float().numpy()[None, :])
+            ref = oracle.group_error(np.ascontiguousarray(y, dtype=np.float32), fmt)
+        else:
+            y = oracle.rotate(synth.bf16_bits(x), block, None if sg is None else synth.bf16_bits(sg))
+            ref = oracle.group_error(y, fmt)
+        check(gpu(bro, x, block, sg, fmt=fmt), ref)
+
+
+def test_largest_magnitudes_without_rotation(bro):
+    """Groups whose maximum is in the top binade of fp32 (reachable only without a rotation): the error
+    itself is beyond fp32 there, and the fp32 statistic has to say so (infinity), not zero."""
+    K = 96
+    x = torch.zeros((1, K), dtype=torch.bfloat16)
+    x[0, 3] = 3e38
+    x[0, 9] = -1.1e38
+    x[0, 40] = 2.5e38
+    x[0, 41] = 1e37
+    x[0, 70] = 1.5
+    x[0, 71] = -0.3
+    for fmt in ("mxfp4", "mxint4", "bfp4", "bint4"):
+        ref = oracle.group_error(np.ascontiguousarray(x.float().numpy()), fmt)
+        got = gpu(bro, x, 1, fmt=fmt)
+        assert np.all(ref[0, :2] > 3.5e38) and np.all(np.isinf(got[0, :2])), (fmt, got, ref)
+        assert abs(got[0, 2] - ref[0, 2]) <= 1e-5 * ref[0, 2]

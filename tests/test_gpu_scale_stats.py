@@ -38,7 +38,7 @@ def test_scale_bytes_all_rotations(bro, M, K):
     x = synth.activations(M, K, seed=M + K)
     bits = synth.bf16_bits(x)
     xd = x.cuda()
-    blocks = [1] + [b for b in (32, 64, 128) if K % b == 0] + ([0] if K & (K - 1) == 0 else [])
+    blocks = [1, 2, 4, 8, 16] + [b for b in (32, 64, 128) if K % b == 0] + ([0] if K & (K - 1) == 0 else [])
     for block in blocks:
         got = gpu_scale_bytes(bro, xd, block).cpu().numpy()
         assert np.array_equal(got, oracle.group_scale_bytes(bits, block)), f"block {block}"
@@ -48,7 +48,7 @@ def test_scale_bytes_all_rotations(bro, M, K):
     assert bro.last_device_status() == 0
 
 
-@pytest.mark.parametrize("block", [1, 32, 64, 128, 0])
+@pytest.mark.parametrize("block", [1, 2, 8, 16, 32, 64, 128, 0])
 def test_scale_bytes_with_a_sign_vector(bro, block):
     """A sign vector changes the rotated values (not their magnitudes under the identity): every rotation
     size against the oracle's randomised rotation."""
@@ -150,7 +150,7 @@ def test_empty_inputs_and_argument_checks(bro):
     x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
     out = torch.zeros((4, 2), dtype=torch.uint8, device="cuda")
     with pytest.raises(bro.BroError):
-        bro.group_scale_bytes(x, 16, out)
+        bro.group_scale_bytes(x, 24, out)          # not a power of two
     ws = torch.empty(16, dtype=torch.uint8, device="cuda")
     with pytest.raises(bro.BroError):
         bro.outlier_groups(x, out, torch.zeros(4, dtype=torch.int32, device="cuda"), ws)
