@@ -108,7 +108,8 @@ bro_status bro_last_device_status_ex(void* stream, int* site);
  * ascending stride order, one multiply by the fp32 nearest 1/sqrt(block) at the end — then each
  * group of 32 values of y is quantised to MXFP4.
  *   block   32, 64 or 128; or 0 for block = K (global rotation; K must then be a power of two,
- *           32 <= K <= 32768).
+ *           32 <= K <= 32768); or 2, 4, 8, 16 — a rotation inside the MX group (Sec. 5.2 sweeps the
+ *           rotation dimension below as well as above the group size; the butterfly stops early).
  *   ldx     row stride of x in elements, >= K, multiple of 8.
  *   codes   out, [M, K/2] bytes, 16-byte aligned.
  *   scales  out, bro_scales_bytes(M, K, layout) bytes, 16-byte aligned.
@@ -164,7 +165,7 @@ bro_status bro_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int
  * paper does not spell the producer out; this is the library's reading).  Then the activation path of
  * bro_rotate_quantize_mxfp4 on h.
  *   gate_bf16, up_bf16  [M, K] bf16, row strides ldg / ldu in elements (>= K, multiples of 8), 16-byte aligned.
- *   block               32, 64 or 128 (block = 0 is not offered here: BRO_ERR_UNSUPPORTED).
+ *   block               2, 4, 8, 16, 32, 64 or 128 (block = 0 is not offered here: BRO_ERR_UNSUPPORTED).
  *   signs_bf16          NULL or the +-1 vector of the randomised rotation.
  * bro_swiglu_bf16 is the producer alone (h as a bf16 tensor [M, ldh]), for callers that need h itself.
  * bro_swiglu_linear is bro_linear(_rs) with the fused producer in front: y = Q(h R) Q(W R)^T.
@@ -196,7 +197,7 @@ typedef struct {
   uint32_t magic;     /* BRO_WEIGHTS_MAGIC */
   uint32_t version;   /* BRO_WEIGHTS_VERSION */
   int64_t N, K;
-  int32_t block;      /* rotation block the weights were packed with: 32, 64, 128 or 0 (= K) */
+  int32_t block;      /* rotation block the weights were packed with: 2 .. 128 or 0 (= K) */
   int32_t randomised; /* 1 if a sign vector was applied */
   const void* codes;  /* device, bro_codes_bytes(N, K) bytes */
   const void* scales; /* device, bro_scales_bytes(N, K, BRO_LAYOUT_GEMM) bytes */
@@ -234,9 +235,7 @@ bro_status bro_linear_rs(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
  * row of x and every group of 32 channels of y = x R_block:
  *   mse[m, g] = mean_i (y_i - deq(Q(y))_i)^2
  * with Q the MXFP4 quantiser of bro_rotate_quantize_mxfp4.  Nothing else is written.
- *   block       32, 64, 128 or 0 (= K), as above; also 1 (no rotation) and 2, 4, 8, 16 (a rotation
- *               inside the MX group: Sec. 5.2 sweeps the rotation dimension below as well as above
- *               the group size; these sizes exist in the analysis calls only);
+ *   block       2, 4, 8, 16, 32, 64, 128 or 0 (= K), as above; also 1 (no rotation);
  *   signs_bf16  NULL or the +-1 vector of the randomised rotation;  mse  device, fp32 [M, K/32], dense.
  * Arithmetic: differences are exact, squares and their sum are rounded in fp32 (relative error of a
  * few 2^-24 against an fp64 evaluation).

@@ -24,6 +24,11 @@ constexpr int64_t kGroup = 32;
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+inline int log2_of(int64_t v) {
+  int lg = 0;
+  while (((int64_t)1 << lg) < v) ++lg;
+  return lg;
+}
 
 // ---- device / driver plumbing ------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -188,7 +193,8 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   if (!x || !codes || !scales) return BRO_ERR_NULL;
   if (layout != BRO_LAYOUT_CANONICAL && layout != BRO_LAYOUT_GEMM) return BRO_ERR_SHAPE;
   const int64_t B = block == 0 ? K : block;
-  if (block != 0 && block != 32 && block != 64 && block != 128) return BRO_ERR_SHAPE;
+  // 32, 64, 128 or K; also 2, 4, 8, 16 — a rotation inside the MX group (Sec. 5.2 sweeps the dimension both ways)
+  if (block != 0 && !(block >= 2 && block <= 128 && is_pow2(block))) return BRO_ERR_SHAPE;
   if (K % B != 0) return BRO_ERR_SHAPE;
   if (block == 0 && (!is_pow2(K) || K < 32 || K > 32768)) return BRO_ERR_UNSUPPORTED;
   if (ldx % 8 != 0 || !aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(signs, 16))
@@ -207,15 +213,19 @@ bro_status launch_rotate_quantize(const void* x, int64_t M, int64_t K, int64_t l
   // large inputs its extra registers cost occupancy and the TMA ring is faster.  The flags of the
   // *_ex entry point override the choice.
   const bool can_direct = bro::rqd::supports(M, K, layout, gemm_scale_kblocks(K));
-  bool direct = can_direct && (B == 32 || M * K <= ((int64_t)1 << 23));
+  bool direct = can_direct && (B <= 32 || M * K <= ((int64_t)1 << 23));
   if (flags & BRO_FLAG_RQ_TMA_RING) direct = false;
   else if (flags & BRO_FLAG_RQ_DIRECT) direct = can_direct;
+  if (B < 32) {                   // blocks below the MX group exist in the register-streaming kernel only
+    if (!can_direct) return BRO_ERR_UNSUPPORTED;
+    direct = true;
+  }
   if (up) {                       // the fused producer exists in the register-streaming kernel only
     if (!can_direct) return BRO_ERR_UNSUPPORTED;
     direct = true;
   }
   if (direct)
-    return bro::rqd::launch(x, M, K, ldx, B == 32 ? 5 : (B == 64 ? 6 : 7), signs, codes, scales, layout,
+    return bro::rqd::launch(x, M, K, ldx, log2_of(B), signs, codes, scales, layout,
                             gemm_scale_kblocks(K), di.sm_count, st, up, ldu);
 
   CUtensorMap tmx;

@@ -115,22 +115,6 @@ struct Params {
   int64_t total_tasks;          // M * chunks_per_row
 };
 
-// Butterfly stages of stride 2 .. B/2 on pairs, for B <= 16 (pair k meets pair k ^ (h/2)).
-template <int LOG2B>
-__device__ __forceinline__ void fwht_small(uint64_t (&P)[16]) {
-#pragma unroll
-  for (int hp = 1; hp < (1 << (LOG2B - 1)); hp <<= 1) {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      if ((k & hp) == 0) {
-        const uint64_t a = P[k], b = P[k + hp];
-        P[k] = rq::add2(a, b);
-        P[k + hp] = rq::sub2(a, b);
-      }
-    }
-  }
-}
-
 // LOG2B = 0: no rotation; 1..4: blocks of 2..16 inside the group; 5, 6, 7: blocks of 32, 64, 128.
 template <int LOG2B, bool SIGNS>
 __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params p) {
@@ -163,7 +147,7 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
       }
     }
     if (LOG2B >= 5) rq::fwht32_stages_2_to_16(P);
-    if (LOG2B >= 2 && LOG2B <= 4) fwht_small<(LOG2B >= 2 && LOG2B <= 4) ? LOG2B : 2>(P);
+    if (LOG2B >= 2 && LOG2B <= 4) rq::fwht32_stages_below<(LOG2B >= 2 && LOG2B <= 4) ? LOG2B : 2>(P);
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
     if (!full) {                                   // the statistics only

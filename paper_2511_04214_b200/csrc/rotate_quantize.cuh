@@ -147,6 +147,24 @@ __device__ __forceinline__ void fwht32_stages_2_to_16(uint64_t (&P)[16]) {
   }
 }
 
+// The same for a rotation inside the MX group (blocks of 2..16 channels: LOG2B = 1..4): the stages of
+// stride 2 .. B/2 only (stage h = 1 is in unpack_stage1).
+template <int LOG2B>
+__device__ __forceinline__ void fwht32_stages_below(uint64_t (&P)[16]) {
+  static_assert(LOG2B >= 1 && LOG2B <= 4, "blocks of 2..16");
+#pragma unroll
+  for (int hp = 1; hp < (1 << (LOG2B - 1)); hp <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      if ((k & hp) == 0) {
+        const uint64_t a = P[k], b = P[k + hp];
+        P[k] = add2(a, b);
+        P[k + hp] = sub2(a, b);
+      }
+    }
+  }
+}
+
 // ---- blocks of 64 / 128 channels: cross-lane stages that exchange HALF of each lane's values --------
 // The 2 (or 4) MX groups of a block sit in neighbouring lanes.  A butterfly stage between two lanes
 // needs, for every element i, a + b in one lane and a - b in the other.  Instead of every lane

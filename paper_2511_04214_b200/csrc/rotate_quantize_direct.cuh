@@ -202,7 +202,8 @@ rotate_quantize_direct_kernel(const Params p) {
       chunk = nchunk;
       continue;
     }
-    rq::fwht32_stages_2_to_16(P);
+    if constexpr (LOG2B >= 5) rq::fwht32_stages_2_to_16(P);
+    else rq::fwht32_stages_below<LOG2B>(P);          // a rotation inside the MX group stops early
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
     if (STATS) {
@@ -277,6 +278,25 @@ inline bro_status launch_one(Params& p, int sm_count, cudaStream_t st) {
 
 template <bool STATS, bool PRODUCER = false>
 inline bro_status launch_any(Params& p, int log2b, int sm_count, cudaStream_t st) {
+  if constexpr (!STATS) {       // rotations inside the MX group (blocks of 2..16): the quantising kernels only
+    if (p.signs) {
+      switch (log2b) {
+        case 1: return launch_one<1, true, false, PRODUCER>(p, sm_count, st);
+        case 2: return launch_one<2, true, false, PRODUCER>(p, sm_count, st);
+        case 3: return launch_one<3, true, false, PRODUCER>(p, sm_count, st);
+        case 4: return launch_one<4, true, false, PRODUCER>(p, sm_count, st);
+        default: break;
+      }
+    } else {
+      switch (log2b) {
+        case 1: return launch_one<1, false, false, PRODUCER>(p, sm_count, st);
+        case 2: return launch_one<2, false, false, PRODUCER>(p, sm_count, st);
+        case 3: return launch_one<3, false, false, PRODUCER>(p, sm_count, st);
+        case 4: return launch_one<4, false, false, PRODUCER>(p, sm_count, st);
+        default: break;
+      }
+    }
+  }
   if (p.signs) {
     switch (log2b) {
       case 5: return launch_one<5, true, STATS, PRODUCER>(p, sm_count, st);

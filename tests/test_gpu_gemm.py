@@ -173,7 +173,7 @@ def test_linear_end_to_end_config1(bro):
     """bro_linear = kernel 1 + kernel 2 on device, against the oracle's whole-layer result."""
     x = synth.activations(64, 2048, seed=0, recipe=synth.CFG1_RECIPE)
     w = synth.weights(2048, 2048, seed=0)
-    for block in (32, 64, 128, 0):
+    for block in (32, 64, 128, 0, 8, 16):          # (8, 16: rotation dimensions below the MX group)
         wc_ref, ws_ref = oracle.pack_weights(synth.bf16_bits(w), block)
         y_ref, S = oracle.linear(synth.bf16_bits(x), block, wc_ref, ws_ref)
         wcodes = bro.alloc_codes(2048, 2048)

@@ -54,6 +54,14 @@ def test_codes_and_scales_bit_exact(bro, form, block, M, K):
     compare(bro, x, signs, block, 0, form)
 
 
+@pytest.mark.parametrize("block", [2, 4, 8, 16])
+def test_rotations_inside_the_mx_group(bro, block):
+    x = synth.activations(129, 416, seed=60 + block)
+    signs = synth.rotation_signs(416, seed=61)
+    compare(bro, x, signs, block, 1)
+    compare(bro, x, signs, block, 0)
+
+
 def test_ragged_k_and_all_plus_signs(bro):
     x = synth.activations(129, 416, seed=2)
     compare(bro, x, synth.rotation_signs(416, seed=3), 32, 1)

@@ -63,6 +63,17 @@ def test_config1_activations(bro, form, block, layout):
     compare(bro, x, block, layout, form)
 
 
+@pytest.mark.parametrize("block", [2, 4, 8, 16])
+@pytest.mark.parametrize("M,K", [(1, 32), (7, 160), (129, 416), (300, 1024), (64, 4096)])
+def test_rotations_inside_the_mx_group(bro, M, K, block):
+    """Rotation dimensions below the MX group (Sec. 5.2 sweeps the dimension both ways): the butterfly of a
+    group stops early; codes and scales bit-exact in both layouts."""
+    x = synth.activations(M, K, seed=900 + M + block)
+    compare(bro, x, block, 1)
+    compare(bro, x, block, 0)
+    compare(bro, x, block, 1, bro.FLAG_RQ_TMA_RING)        # (the flag has no say at these sizes)
+
+
 RAGGED = [(M, K, b) for (M, K) in [(1, 32), (1, 128), (7, 160), (129, 416), (300, 1024), (513, 2176), (1024, 4096)]
           for b in (32, 64, 128) if K % b == 0]
 
