@@ -79,8 +79,8 @@ NCU_TRAFFIC = {
              "per_row_of": (8192, 8192, 28672), "bytes": 535339776 + 441953536},
     "cfg3": {"sources": GEMM_SOURCES, "digest": "096c61cb1b9865ca985e775b0d340c5efb1060c2d39547c30f96dd9d3d65fab1",
              "shapes": {(4096, 4096, 14336): 68345088 + 69353728}},
-    "cfg4": {"sources": RQ_SOURCES, "digest": "2d3859b1f32f3f300839f554c09980e668d03fc390304cf7692f4ce40247a6d2",
-             "shapes": {(16384, 4096, 32): 134230784 + 19085312}},
+    "cfg4": {"sources": RQ_SOURCES, "digest": "aa6e030cc76b05e3c4883ecbdfdbfc516261469c9425d0325a4fb2e97853c75c",
+             "shapes": {(16384, 4096, 32): 134233600 + 19132928}},
 }
 
 

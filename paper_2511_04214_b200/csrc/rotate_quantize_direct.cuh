@@ -14,7 +14,8 @@
 // warps are resident and they drift apart, so loads, arithmetic and stores of different warps
 // overlap.  Blocks of 64 / 128 channels pair lanes l ^ 1 (and l ^ 2) for their last one / two stages,
 // each lane exchanging half of its values (rq::cross_lane_split); the per-group error kernels keep the
-// whole group in one lane (rq::cross_lane_stage).
+// whole group in one lane (rq::cross_lane_stage).  Blocks of 2..16 channels (a rotation inside the MX
+// group, LOG2B = 1..4) stop the butterfly early (rq::fwht32_stages_below).
 #pragma once
 
 #include "bro_common.cuh"
