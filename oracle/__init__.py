@@ -227,7 +227,7 @@ def group_mse(y, codes, scales) -> np.ndarray:
     return mse
 
 
-FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3}
+FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3, "int4_row_sym": 4, "int4_row_asym": 5}
 
 
 def fake_quantize(y, fmt) -> np.ndarray:

@@ -325,9 +325,56 @@ static float round_to_fp16(float f) {
   return f < 0 ? -a : a;
 }
 
+/* INT4 with one scale per ROW (Sec. 3.2 / Fig. 2: "INT4 — weight per-channel symmetric quantization with
+ * per-token asymmetric activation quantization"): format 4 is the symmetric form (a row of W is an output
+ * channel), format 5 the asymmetric form (a row of X is a token). */
+static void int4_row(const float* v, int64_t K, int asym, double* out) {
+  if (!asym) {
+    float amax = 0.0f;
+    for (int64_t i = 0; i < K; ++i)
+      if (fabsf(v[i]) > amax) amax = fabsf(v[i]);
+    const float sc = round_to_fp16(amax / 7.0f);
+    for (int64_t i = 0; i < K; ++i) {
+      if (sc == 0.0f) { out[i] = 0.0; continue; }
+      double q = rint((double)(fabsf(v[i]) / sc)); /* fp32 division, ties to even */
+      if (q > 7.0) q = 7.0;
+      q *= (double)sc;
+      out[i] = (f32_bits(v[i]) >> 31) ? -q : q;
+    }
+    return;
+  }
+  /* the range always contains zero, so that zero stays exactly representable */
+  float lo = 0.0f, hi = 0.0f;
+  for (int64_t i = 0; i < K; ++i) {
+    if (v[i] < lo) lo = v[i];
+    if (v[i] > hi) hi = v[i];
+  }
+  const float sc = round_to_fp16((hi - lo) / 15.0f); /* fp32 subtraction and division, then fp16 */
+  if (sc == 0.0f) {
+    for (int64_t i = 0; i < K; ++i) out[i] = 0.0;
+    return;
+  }
+  double z = rint((double)(-lo / sc)); /* zero point: the code of 0.0 */
+  if (z > 15.0) z = 15.0;
+  for (int64_t i = 0; i < K; ++i) {
+    double q = rint((double)(v[i] / sc));
+    if (q > 31.0) q = 31.0;
+    if (q < -16.0) q = -16.0;
+    q += z;
+    if (q > 15.0) q = 15.0;
+    if (q < 0.0) q = 0.0;
+    out[i] = (q - z) * (double)sc;
+  }
+}
+
 int bro_ref_fake_quantize(const float* y, int64_t rows, int64_t K, int format, double* deq) {
   if (!y || !deq) return 1;
-  if (rows < 0 || K <= 0 || K % MX_GROUP != 0 || format < 0 || format > 3) return 2;
+  if (rows < 0 || K <= 0 || K % MX_GROUP != 0 || format < 0 || format > 5) return 2;
+  if (format >= 4) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) int4_row(y + r * K, K, format == 5, deq + r * K);
+    return 0;
+  }
   const int64_t ng = K / MX_GROUP;
 #pragma omp parallel for schedule(static)
   for (int64_t r = 0; r < rows; ++r)

@@ -113,6 +113,12 @@ int bro_ref_group_mse(const float* y, const uint8_t* codes, const uint8_t* scale
  *   1 BFP4    E2M1 elements, FP16 scale s = fp16(amax / 6)                       ("FP4 variant of BINT4")
  *   2 MXINT4  INT4 elements k/4, k in [-7, 7], E8M0 scale 2^E, E = floor(log2 amax)
  *   3 BINT4   INT4 elements k in [-7, 7], FP16 scale s = fp16(amax / 7)          (RTN, block 32, FP16 scale)
+ * and INT4 with one scale per ROW of y instead of per group (Sec. 3.2 / Fig. 2: per-channel symmetric
+ * for weights, per-token asymmetric for activations):
+ *   4 INT4 row, symmetric    k in [-7, 7], s = fp16(amax_row / 7)
+ *   5 INT4 row, asymmetric   codes q in [0, 15] over the range [lo, hi] = [min(row, 0), max(row, 0)]:
+ *                            s = fp16((hi - lo) / 15), zero point z = rint(-lo / s) (clamped to 15),
+ *                            q = clamp(rint(y / s) + z, 0, 15), dequantised (q - z) s
  * The paper names the formats but gives no formulas; the scale and rounding rules above are this
  * build's reading (round to nearest even everywhere, saturating; fp16 scale = the fp32 quotient
  * rounded to nearest-even fp16, clamped to the largest finite fp16; a zero scale gives all zeros).
