@@ -587,23 +587,24 @@ def block_sweep(bro, synth, peaks, blocks, groups):
     # Simulated quantisation (Sec. 3.1: how the paper evaluates the formats): rotate, quantise, dequantise
     # to fp32 in one launch — 2 B read and 4 B written per element.
     deq = torch.empty((M, K), dtype=torch.float32, device="cuda")
+    fws = torch.empty(bro.fake_quantize_workspace_bytes(M, "int4_row_asym"), dtype=torch.uint8, device="cuda")
     fake = {}
-    for fmt in ("mxfp4", "bfp4", "mxint4", "bint4"):
+    for fmt in ("mxfp4", "bfp4", "mxint4", "bint4", "int4_row_sym", "int4_row_asym"):     # (the last two: two passes over x)
         for i in range(2):
-            bro.rotate_fake_quantize(xs[i % ring], 32, deq, fmt)
+            bro.rotate_fake_quantize(xs[i % ring], 32, deq, fmt, workspace=fws)
         ts = []
         for gi in range(max(2, groups // 2)):
             a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for i in range(ring):
-                bro.rotate_fake_quantize(xs[i % ring], 32, deq, fmt)
+                bro.rotate_fake_quantize(xs[i % ring], 32, deq, fmt, workspace=fws)
             c.record()
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(c) / ring)
         ms = statistics.mean(ts)
         fake[fmt] = {"us": round(ms * 1e3, 2), "gbs": round(M * K * 6.0 / (ms * 1e-3) / 1e9, 1),
                      "frac_of_measured_copy": round(M * K * 6.0 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
-    del deq
+    del deq, fws
     return {"shape_MK": [M, K], "algorithmic_bytes": bytes_per_launch, "per_block": per_block,
             "swiglu_producer_block32": producer, "fake_quantize_block32": fake,
             "timing": f"CUDA events around groups of {group} back-to-back launches, {groups} groups per size"}, (xs, codes, scales)

@@ -73,7 +73,11 @@ typedef enum {
 typedef enum { BRO_LAYOUT_CANONICAL = 0, BRO_LAYOUT_GEMM = 1 } bro_layout;
 typedef enum { BRO_OUT_BF16 = 0, BRO_OUT_F32 = 1 } bro_out_dtype;
 /* 4-bit formats of the analysis entry point (see bro_group_quant_error_fmt). */
-typedef enum { BRO_FMT_MXFP4 = 0, BRO_FMT_BFP4 = 1, BRO_FMT_MXINT4 = 2, BRO_FMT_BINT4 = 3 } bro_format;
+typedef enum {
+  BRO_FMT_MXFP4 = 0, BRO_FMT_BFP4 = 1, BRO_FMT_MXINT4 = 2, BRO_FMT_BINT4 = 3,
+  /* bro_rotate_fake_quantize(_ws) only: INT4 with one scale per row, and no quantisation at all */
+  BRO_FMT_INT4_ROW_SYM = 4, BRO_FMT_INT4_ROW_ASYM = 5, BRO_FMT_NONE = 6
+} bro_format;
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* bro_status_string(bro_status s);
@@ -279,6 +283,28 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
 bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
                                     const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
                                     void* stream);
+/*
+ * The same with a workspace, which opens three more values of `format`:
+ *   BRO_FMT_INT4_ROW_SYM   INT4 with one scale per ROW, symmetric: |k| <= 7, scale fp16(amax_row / 7)
+ *   BRO_FMT_INT4_ROW_ASYM  INT4 with one scale per row, asymmetric: codes q in [0, 15] over the range
+ *                          [lo, hi] = [min(row, 0), max(row, 0)], scale s = fp16((hi - lo) / 15), zero
+ *                          point z = rint(-lo / s) (at most 15), q = clamp(rint(y / s) + z, 0, 15),
+ *                          dequantised (q - z) s
+ *   BRO_FMT_NONE           no quantisation: deq = x diag(s) R_block itself, the fp32 values every other
+ *                          format is an approximation of (so that the caller can form any error statistic)
+ * The first two are the fifth format of the paper's study (Sec. 3.2 / Fig. 2: "INT4" = per-channel
+ * symmetric weights — a row of W is an output channel — and per-token asymmetric activations — a row
+ * of X is a token); the paper gives no formulas, the rules above are this library's reading.  They
+ * take two passes over x (the first leaves each row's range in the workspace) and need
+ *   workspace   device, bro_fake_quantize_workspace_bytes(M, format) bytes (8 per row; 0 for the other
+ *               formats, which ignore it), 8-byte aligned; contents undefined afterwards.
+ * BRO_ERR_WORKSPACE if it is missing or too small.  bro_rotate_fake_quantize is this call without a
+ * workspace.  Everything else as above.
+ */
+size_t bro_fake_quantize_workspace_bytes(int64_t M, bro_format format);
+bro_status bro_rotate_fake_quantize_ws(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                       const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
+                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Scale statistics behind the paper's regular-block / outlier-block argument (Sec. 4.1: "regular

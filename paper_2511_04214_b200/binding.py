@@ -25,7 +25,7 @@ EXPORTS = [
     "bro_gemm_workspace_bytes", "bro_linear_workspace_bytes", "bro_last_device_status",
     "bro_rotate_quantize_mxfp4", "bro_pack_weights", "bro_gemm_mxfp4", "bro_linear",
     "bro_linear_host", "bro_linear_static",
-    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt", "bro_rotate_fake_quantize",
+    "bro_rotate_quantize_mxfp4_rs", "bro_pack_weights_rs", "bro_linear_rs", "bro_group_quant_error", "bro_group_quant_error_fmt", "bro_rotate_fake_quantize", "bro_rotate_fake_quantize_ws", "bro_fake_quantize_workspace_bytes",
     "bro_last_device_status_ex", "bro_selftest_expire_wait",
     "bro_rotate_quantize_mxfp4_ex", "bro_gemm_mxfp4_ex", "bro_linear_ex",
     "bro_group_scale_bytes", "bro_outlier_workspace_bytes", "bro_outlier_groups", "bro_scale_histogram",
@@ -103,6 +103,10 @@ def _load() -> ctypes.CDLL:
     L.bro_group_quant_error_fmt.argtypes = [p, i64, i64, i64, ci, p, ci, p, p]
     L.bro_rotate_fake_quantize.restype = ci
     L.bro_rotate_fake_quantize.argtypes = [p, i64, i64, i64, ci, p, ci, p, i64, p]
+    L.bro_rotate_fake_quantize_ws.restype = ci
+    L.bro_rotate_fake_quantize_ws.argtypes = [p, i64, i64, i64, ci, p, ci, p, i64, p, sz, p]
+    L.bro_fake_quantize_workspace_bytes.restype = sz
+    L.bro_fake_quantize_workspace_bytes.argtypes = [i64, ci]
     L.bro_linear_static.restype = ci
     L.bro_linear_static.argtypes = [p, i64, i64, i64, ci, p, p, i64, p, i64, p]
     L.bro_group_scale_bytes.restype = ci
@@ -328,7 +332,7 @@ def linear_rs(x: torch.Tensor, block: int, signs: torch.Tensor, wcodes, wscales,
            "bro_linear_rs")
 
 
-FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3}
+FORMATS = {"mxfp4": 0, "bfp4": 1, "mxint4": 2, "bint4": 3, "int4_row_sym": 4, "int4_row_asym": 5, "none": 6}
 
 
 def group_quant_error(x: torch.Tensor, block: int, mse: torch.Tensor, signs: torch.Tensor = None,
@@ -341,15 +345,22 @@ def group_quant_error(x: torch.Tensor, block: int, mse: torch.Tensor, signs: tor
                                          _stream(stream)), "bro_group_quant_error_fmt")
 
 
+def fake_quantize_workspace_bytes(M: int, fmt: str) -> int:
+    return int(lib.bro_fake_quantize_workspace_bytes(M, FORMATS[fmt]))
+
+
 def rotate_fake_quantize(x: torch.Tensor, block: int, deq: torch.Tensor, fmt: str = "mxfp4", signs: torch.Tensor = None,
-                         stream=None) -> None:
+                         workspace: torch.Tensor = None, stream=None) -> None:
     """Simulated quantisation: ``deq`` (fp32 [M, K], rows may be strided) receives the dequantised values of
-    x R_block quantised to ``fmt``; block = 1: no rotation, 0: the full dimension."""
+    x R_block quantised to ``fmt``; block = 1: no rotation, 0: the full dimension.  The per-row formats
+    ("int4_row_sym", "int4_row_asym") need ``workspace`` (fake_quantize_workspace_bytes); "none" returns the
+    rotated values themselves."""
     assert x.dtype == torch.bfloat16 and deq.dtype == torch.float32
     M, K = x.shape
     assert deq.shape == (M, K)
-    _check(lib.bro_rotate_fake_quantize(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(deq), _ld(deq, K),
-                                        _stream(stream)), "bro_rotate_fake_quantize")
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.bro_rotate_fake_quantize_ws(_ptr(x), M, K, _ld(x, K), block, _ptr(signs), FORMATS[fmt], _ptr(deq), _ld(deq, K),
+                                           _ptr(workspace), wbytes, _stream(stream)), "bro_rotate_fake_quantize_ws")
 
 
 def group_scale_bytes(x: torch.Tensor, block: int, scales: torch.Tensor, signs: torch.Tensor = None, stream=None) -> None:

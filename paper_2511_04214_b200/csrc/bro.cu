@@ -400,10 +400,15 @@ bro_status bro_group_quant_error_fmt(const void* x_bf16, int64_t M, int64_t K, i
 }
 
 // ---- simulated quantisation ----------------------------------------------------------------------
-bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
-                                    const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
-                                    void* stream) {
-  if ((int)format < 0 || (int)format > 3) return BRO_ERR_SHAPE;
+size_t bro_fake_quantize_workspace_bytes(int64_t M, bro_format format) {
+  const bool rows = format == BRO_FMT_INT4_ROW_SYM || format == BRO_FMT_INT4_ROW_ASYM;
+  return (rows && M > 0) ? (size_t)M * 8 : 0;
+}
+
+bro_status bro_rotate_fake_quantize_ws(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                       const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  if ((int)format < 0 || (int)format > (int)BRO_FMT_NONE) return BRO_ERR_SHAPE;
   if (M < 0 || K <= 0 || K % kGroup != 0 || ldx < K || ldd < K) return BRO_ERR_SHAPE;
   if (M > (int64_t)1 << 30 || K > (int64_t)1 << 30) return BRO_ERR_SHAPE;
   if (!analysis_block(block)) return BRO_ERR_SHAPE;
@@ -414,14 +419,34 @@ bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, in
   if (!x_bf16 || !deq) return BRO_ERR_NULL;
   if (ldx % 8 != 0 || ldd % 4 != 0 || !aligned(x_bf16, 16) || !aligned(deq, 16) || !aligned(signs_bf16, 16))
     return BRO_ERR_ALIGN;
+  const size_t need = bro_fake_quantize_workspace_bytes(M, format);
+  if (need > 0 && (!workspace || workspace_bytes < need)) return BRO_ERR_WORKSPACE;
+  if (need > 0 && !aligned(workspace, 8)) return BRO_ERR_ALIGN;
   DeviceInfo di;
   bro_status rc = device_info(&di);
   if (rc != BRO_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* rowstats = need > 0 ? static_cast<uint32_t*>(workspace) : nullptr;
+  if (rowstats) {
+    // per-row formats: a first pass leaves every row's range in the workspace
+    if (!bro::cuda_ok(cudaMemsetAsync(rowstats, 0, need, st), "cudaMemsetAsync(row ranges)")) return BRO_ERR_CUDA;
+    rc = B > 128 ? bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, nullptr, (int)format, BRO_LAYOUT_CANONICAL,
+                                    0, di.sm_count, st, nullptr, 0, rowstats, true)
+                 : bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, nullptr, 0, nullptr, nullptr,
+                                   di.sm_count, st, rowstats);
+    if (rc != BRO_OK) return rc;
+  }
   if (B > 128)
     return bro::rqg::launch(x_bf16, M, K, ldx, signs_bf16, nullptr, nullptr, nullptr, (int)format, BRO_LAYOUT_CANONICAL, 0,
-                            di.sm_count, st, deq, ldd);
-  return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, deq, ldd, nullptr, nullptr, di.sm_count, st);
+                            di.sm_count, st, deq, ldd, rowstats, false);
+  return bro::fq::launch(x_bf16, M, K, ldx, (int)B, signs_bf16, (int)format, deq, ldd, nullptr, nullptr, di.sm_count, st,
+                         rowstats);
+}
+
+bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, int block,
+                                    const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
+                                    void* stream) {
+  return bro_rotate_fake_quantize_ws(x_bf16, M, K, ldx, block, signs_bf16, format, deq, ldd, nullptr, 0, stream);
 }
 
 // ---- scale statistics ----------------------------------------------------------------------------

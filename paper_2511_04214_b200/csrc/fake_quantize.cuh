@@ -102,10 +102,71 @@ __device__ __forceinline__ void store_group(float* dst, const float (&out)[32]) 
     reinterpret_cast<float4*>(dst)[j] = make_float4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
 }
 
+// ---- INT4 with one scale per ROW (Sec. 3.2 / Fig. 2: per-channel symmetric weights, per-token asymmetric
+// activations).  Two passes over the input: the first leaves the row's range in `rowstats`, the second
+// quantises with it.  rowstats[2 * row] = bits of max(-min(row), 0), rowstats[2 * row + 1] = bits of
+// max(max(row), 0): both are non-negative floats, which order like their bit patterns, so an integer
+// atomicMax onto zero-initialised words is an exact, order-independent reduction.
+constexpr int kFormatRowSym = 4, kFormatRowAsym = 5, kFormatNone = 6;
+
+__device__ __forceinline__ void group_range(const uint64_t (&P)[16], uint32_t cbits, float& neglo, float& hi) {
+  const float c = __uint_as_float(cbits);
+  const uint64_t cc = rq::pack2(c, c);
+  neglo = 0.f;
+  hi = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    float a, b;
+    rq::unpack2(rq::mul2(P[k], cc), a, b);
+    hi = fmaxf(hi, fmaxf(a, b));
+    neglo = fmaxf(neglo, fmaxf(-a, -b));
+  }
+}
+
+// The 32 values of a group under the row's scale.  Symmetric: |k| <= 7, scale fp16(amax / 7).  Asymmetric:
+// codes 0..15 over [lo, hi] (the range always contains zero): scale fp16((hi - lo) / 15), zero point
+// z = rint(-lo / scale) (at most 15), q = clamp(rint(y / scale) + z, 0, 15), value (q - z) scale.  Quotients
+// are IEEE fp32 divisions; every result is an integer of at most 5 bits times an fp16 number, exact in fp32.
+__device__ __forceinline__ void row_dequant(const uint64_t (&P)[16], uint32_t cbits, bool asym, float neglo, float hi,
+                                            float (&out)[32]) {
+  const float c = __uint_as_float(cbits);
+  const uint64_t cc = rq::pack2(c, c);
+  float y[32];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) rq::unpack2(rq::mul2(P[k], cc), y[2 * k], y[2 * k + 1]);
+  const float quot = asym ? __fdiv_rn(__fadd_rn(hi, neglo), 15.f) : __fdiv_rn(fmaxf(hi, neglo), 7.f);
+  unsigned short hb;
+  asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(hb) : "f"(quot));
+  const float sc = __half2float(__ushort_as_half(hb));
+  if (sc == 0.f) {                  // (a scale that rounds to zero gives an all-zero row)
+#pragma unroll
+    for (int i = 0; i < 32; ++i) out[i] = 0.f;
+    return;
+  }
+  if (!asym) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float q = (float)min(__float2int_rn(__fdiv_rn(fabsf(y[i]), sc)), 7);
+      out[i] = copysignf(__fmul_rn(q, sc), y[i]);
+    }
+    return;
+  }
+  const int z = min(__float2int_rn(__fdiv_rn(neglo, sc)), 15);
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    int q = __float2int_rn(__fdiv_rn(y[i], sc));
+    q = max(-16, min(q, 31)) + z;
+    q = max(0, min(q, 15));
+    out[i] = __fmul_rn((float)(q - z), sc);
+  }
+}
+
 struct Params {
   const uint16_t* x;
   int64_t M, K, ldx;
   const uint16_t* signs;        // [K] bf16 +-1 (kernels with SIGNS) or nullptr
+  uint32_t* rowstats;           // [M, 2] the row ranges (see group_range): written when deq == nullptr and
+                                // neither statistic is asked for, read by the per-row formats
   float* deq;                   // [M, K] fp32, row stride ldd — or nullptr, and then one of:
   int64_t ldd;
   float* mse;                   //   [M, K/32] per-group quantisation error (rq::group_error)
@@ -150,6 +211,20 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
     if (LOG2B >= 2 && LOG2B <= 4) rq::fwht32_stages_below<(LOG2B >= 2 && LOG2B <= 4) ? LOG2B : 2>(P);
     if (LOG2B >= 6) rq::cross_lane_stage(P, 1, (lane & 1) != 0);
     if (LOG2B >= 7) rq::cross_lane_stage(P, 2, (lane & 2) != 0);
+    if (!full && !p.mse && !p.scale_bytes) {       // first pass of the per-row formats: the row's range
+      float neglo, hi;
+      group_range(P, cbits, neglo, hi);
+#pragma unroll
+      for (int d = 16; d >= 1; d >>= 1) {          // (all 32 lanes hold groups of the same row; dead lanes hold zeros)
+        neglo = fmaxf(neglo, __shfl_xor_sync(0xFFFFFFFFu, neglo, d));
+        hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, d));
+      }
+      if (lane == 0) {
+        atomicMax(p.rowstats + 2 * row, __float_as_uint(neglo));
+        atomicMax(p.rowstats + 2 * row + 1, __float_as_uint(hi));
+      }
+      continue;
+    }
     if (!full) {                                   // the statistics only
       if (p.mse) {
         const float e = rq::group_error(P, cbits, p.format);
@@ -161,7 +236,17 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
       continue;
     }
     float out[32];
-    group_dequant(P, cbits, p.format, out);
+    if (p.format == kFormatNone) {                 // the rotation itself
+      const uint64_t cc = rq::pack2(__uint_as_float(cbits), __uint_as_float(cbits));
+#pragma unroll
+      for (int k = 0; k < 16; ++k) rq::unpack2(rq::mul2(P[k], cc), out[2 * k], out[2 * k + 1]);
+    } else if (p.format >= kFormatRowSym) {
+      const float neglo = __uint_as_float(__ldcg(p.rowstats + 2 * row));
+      const float hi = __uint_as_float(__ldcg(p.rowstats + 2 * row + 1));
+      row_dequant(P, cbits, p.format == kFormatRowAsym, neglo, hi, out);
+    } else {
+      group_dequant(P, cbits, p.format, out);
+    }
     // lane l -> buffer row l (128 bytes), piece j at position j ^ (l & 7)
     __syncwarp();                                  // the previous task's reads of the buffer are done
 #pragma unroll
@@ -181,10 +266,13 @@ __global__ void __launch_bounds__(kThreads, 2) fake_quantize_kernel(const Params
   }
 }
 
-// block: 1 (identity), 2, 4, 8, 16, 32, 64 or 128.  Exactly one of deq / mse / scale_bytes is set.
+// block: 1 (identity), 2, 4, 8, 16, 32, 64 or 128.  Exactly one of deq / mse / scale_bytes is set — or none of
+// them and rowstats, for the first pass of the per-row formats.
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, int block, const void* signs, int format,
-                         float* deq, int64_t ldd, float* mse, uint8_t* scale_bytes, int sm_count, cudaStream_t st) {
+                         float* deq, int64_t ldd, float* mse, uint8_t* scale_bytes, int sm_count, cudaStream_t st,
+                         uint32_t* rowstats = nullptr) {
   Params p;
+  p.rowstats = rowstats;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M; p.K = K; p.ldx = ldx;
   p.signs = static_cast<const uint16_t*>(signs);

@@ -32,6 +32,8 @@ struct Params {
   int format;            // ... for this 4-bit format (see rq::group_error)
   float* deq;            // if set: write the dequantised values [M, K] (row stride ldd) under `format` instead
   int64_t ldd;
+  uint32_t* rowstats;    // per-row formats: the row ranges (fq::group_range); written when `range_pass` is set
+  int range_pass;
 };
 
 template <int kMaxThreads>
@@ -97,7 +99,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
         P[2 * c + 1] = rq::pack2(__fmaf_rn(a2, sgn, o.z), __fmaf_rn(a3, sgn, o.w));
       }
     }
-    if (p.format == rq::kFormatScaleOnly) {   // analysis mode (uniform over the grid): scale byte only
+    if (p.format == rq::kFormatScaleOnly && !p.deq && !p.range_pass) {   // analysis mode (uniform over the grid): scale byte only
       const uint32_t sbyte = rq::group_scale_byte(P, cbits);
       if (live) p.scales[row * (p.K >> 5) + gi] = (uint8_t)sbyte;
       continue;
@@ -107,8 +109,26 @@ __global__ void __launch_bounds__(kMaxThreads, 1) rotate_quantize_global_kernel(
       if (live) p.mse[row * (p.K >> 5) + gi] = e;
       continue;
     }
+    if (p.range_pass) {          // first pass of the per-row formats (uniform over the grid)
+      float neglo, hi;
+      fq::group_range(P, cbits, neglo, hi);
+      if (live) {
+        atomicMax(p.rowstats + 2 * row, __float_as_uint(neglo));
+        atomicMax(p.rowstats + 2 * row + 1, __float_as_uint(hi));
+      }
+      continue;
+    }
     if (p.deq) {                 // simulated quantisation (uniform over the grid)
       float out[32];
+      if (p.format == fq::kFormatNone) {
+        const uint64_t cc = rq::pack2(__uint_as_float(cbits), __uint_as_float(cbits));
+#pragma unroll
+        for (int k = 0; k < 16; ++k) rq::unpack2(rq::mul2(P[k], cc), out[2 * k], out[2 * k + 1]);
+      } else if (p.format >= fq::kFormatRowSym) {
+        const int64_t r = live ? row : 0;
+        fq::row_dequant(P, cbits, p.format == fq::kFormatRowAsym, __uint_as_float(__ldcg(p.rowstats + 2 * r)),
+                        __uint_as_float(__ldcg(p.rowstats + 2 * r + 1)), out);
+      } else
       fq::group_dequant(P, cbits, p.format, out);
       if (live) fq::store_group(p.deq + row * p.ldd + (int64_t)gi * 32, out);
       continue;
@@ -347,10 +367,12 @@ bro_status make_row_map(CUtensorMap* map, const void* x, int64_t M, int64_t K, i
 
 inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const void* signs, void* codes,
                          void* scales, float* mse, int format, bro_layout layout, int64_t scale_kblocks, int sm_count, cudaStream_t st,
-                         float* deq = nullptr, int64_t ldd = 0) {
+                         float* deq = nullptr, int64_t ldd = 0, uint32_t* rowstats = nullptr, bool range_pass = false) {
   Params p;
   p.deq = deq;
   p.ldd = ldd;
+  p.rowstats = rowstats;
+  p.range_pass = range_pass ? 1 : 0;
   p.x = static_cast<const uint16_t*>(x);
   p.M = M;
   p.K = K;
@@ -369,12 +391,12 @@ inline bro_status launch(const void* x, int64_t M, int64_t K, int64_t ldx, const
   int threads = p.threads_per_row < 256 ? 256 : p.threads_per_row;
   p.rows_per_iter = threads / p.threads_per_row;
   const size_t smem = K > 1024 ? (size_t)p.rows_per_iter * K * sizeof(float) : 0;
-  if (layout == BRO_LAYOUT_GEMM && !mse && !deq && format != rq::kFormatScaleOnly) {
+  if (layout == BRO_LAYOUT_GEMM && !mse && !deq && !range_pass && format != rq::kFormatScaleOnly) {
     // padding rows / groups of the tiled scale buffer must read as 0
     const size_t bytes = (size_t)((M + 127) / 128) * (size_t)scale_kblocks * 512;
     if (cudaMemsetAsync(scales, 0, bytes, st) != cudaSuccess) return BRO_ERR_CUDA;
   }
-  if ((K == 2048 || K == 4096) && !mse && !deq && format != rq::kFormatScaleOnly) {
+  if ((K == 2048 || K == 4096) && !mse && !deq && !range_pass && format != rq::kFormatScaleOnly) {
     // codes path at these sizes: all stages in registers, two shared-memory transposes
     const int rows = (int)(128 / (K / 32));
     const int64_t iters2 = (M + rows - 1) / rows;

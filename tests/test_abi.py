@@ -103,7 +103,14 @@ def test_fake_quantize_argument_validation_needs_no_device(lib):
     fq = L.bro_rotate_fake_quantize
     assert fq(None, 1, 64, 64, 32, None, 0, p(a16), 64, None) == 1
     assert fq(p(a16), 1, 64, 64, 32, None, 0, None, 64, None) == 1
-    assert fq(p(a16), 1, 64, 64, 32, None, 4, p(a16), 64, None) == 2         # no such format
+    assert fq(p(a16), 1, 64, 64, 32, None, 7, p(a16), 64, None) == 2         # no such format
+    assert fq(p(a16), 1, 64, 64, 32, None, 4, p(a16), 64, None) == 5         # the per-row formats need a workspace
+    ws = L.bro_rotate_fake_quantize_ws
+    assert L.bro_fake_quantize_workspace_bytes(100, 4) == 800 and L.bro_fake_quantize_workspace_bytes(100, 5) == 800
+    assert L.bro_fake_quantize_workspace_bytes(100, 0) == 0 and L.bro_fake_quantize_workspace_bytes(100, 6) == 0
+    assert ws(p(a16), 2, 64, 64, 32, None, 5, p(a16), 64, p(a16), 15, None) == 5       # too small
+    assert ws(p(a16), 2, 64, 64, 32, None, 5, p(a16), 64, p(a16 + 4), 16, None) == 3   # not 8-byte aligned
+    assert ws(p(a16), 0, 64, 64, 32, None, 5, p(a16), 64, None, 0, None) == 0          # no rows: nothing to do
     assert fq(p(a16), 1, 48, 48, 32, None, 0, p(a16), 48, None) == 2         # K not a multiple of 32
     assert fq(p(a16), 1, 96, 96, 24, None, 0, p(a16), 96, None) == 2         # no such block
     assert fq(p(a16), 1, 256, 256, 256, None, 0, p(a16), 256, None) == 2

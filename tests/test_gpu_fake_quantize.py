@@ -12,7 +12,7 @@ from paper_2511_04214_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-FORMATS = ["mxfp4", "bfp4", "mxint4", "bint4"]
+FORMATS = ["mxfp4", "bfp4", "mxint4", "bint4", "int4_row_sym", "int4_row_asym"]
 
 
 @pytest.fixture(scope="module")
@@ -33,7 +33,8 @@ def gpu(bro, x, block, fmt, signs=None, ldd=None):
     M, K = x.shape
     ldd = K if ldd is None else ldd
     buf = torch.full((M, ldd), float("nan"), dtype=torch.float32, device="cuda")
-    bro.rotate_fake_quantize(x.cuda(), block, buf[:, :K], fmt, None if signs is None else signs.cuda())
+    ws = torch.full((bro.fake_quantize_workspace_bytes(M, fmt) + 8,), 0xAB, dtype=torch.uint8, device="cuda")   # (dirty on purpose)
+    bro.rotate_fake_quantize(x.cuda(), block, buf[:, :K], fmt, None if signs is None else signs.cuda(), workspace=ws)
     assert bro.last_device_status() == 0
     out = buf.cpu().numpy()
     assert np.isnan(out[:, K:]).all()              # nothing beyond column K is written
@@ -70,7 +71,8 @@ def test_row_strides_and_untouched_padding(bro, fmt):
     x = big[:, :K]                                  # ldx = K + 64
     xs = big.cuda()[:, :K]
     buf = torch.full((M, K + 12), float("nan"), dtype=torch.float32, device="cuda")
-    bro.rotate_fake_quantize(xs, 64, buf[:, :K], fmt)
+    ws = torch.empty(bro.fake_quantize_workspace_bytes(M, fmt) + 8, dtype=torch.uint8, device="cuda")
+    bro.rotate_fake_quantize(xs, 64, buf[:, :K], fmt, workspace=ws)
     out = buf.cpu().numpy()
     assert np.isnan(out[:, K:]).all()
     check(np.ascontiguousarray(out[:, :K]), oracle.fake_quantize(rotated(x.contiguous(), 64), fmt))
@@ -105,6 +107,26 @@ def test_mxfp4_agrees_with_the_codes_the_gemm_reads(bro):
     assert np.array_equal(got.astype(np.float64), np.asarray(deq, dtype=np.float64))
 
 
+@pytest.mark.parametrize("block,M,K", [(1, 37, 416), (8, 37, 416), (32, 300, 1024), (128, 37, 640), (0, 37, 512), (0, 9, 4096)])
+def test_no_quantisation_returns_the_rotation_itself(bro, block, M, K):
+    """BRO_FMT_NONE: the fp32 rotated values, bit for bit the oracle's rotation."""
+    x = synth.activations(M, K, seed=800 + block)
+    signs = synth.rotation_signs(K, seed=801)
+    for sg in (None, signs):
+        got = gpu(bro, x, block, "none", sg)
+        ref = rotated(x, block, sg)
+        assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(ref, dtype=np.float32).view(np.uint32))
+
+
+def test_row_formats_need_their_workspace(bro):
+    x = synth.activations(4, 64, seed=1).cuda()
+    out = torch.empty((4, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(bro.BroError):
+        bro.rotate_fake_quantize(x, 32, out, "int4_row_asym")
+    with pytest.raises(bro.BroError):
+        bro.rotate_fake_quantize(x, 32, out, "int4_row_sym", workspace=torch.empty(31, dtype=torch.uint8, device="cuda"))
+
+
 def test_full_size_sample(bro):
     """The block-sweep tensor [16384, 4096]: every format at block 32 on sampled rows."""
     M, K = 16384, 4096
@@ -112,8 +134,9 @@ def test_full_size_sample(bro):
     rows = np.unique(np.concatenate([np.arange(0, 8), np.arange(M - 8, M), np.random.default_rng(1).integers(0, M, 48)]))
     xd = x.cuda()
     out = torch.empty((M, K), dtype=torch.float32, device="cuda")
+    ws = torch.empty(8 * M, dtype=torch.uint8, device="cuda")
     for fmt in FORMATS:
-        bro.rotate_fake_quantize(xd, 32, out, fmt)
+        bro.rotate_fake_quantize(xd, 32, out, fmt, workspace=ws)
         got = out[torch.as_tensor(rows, device="cuda")].cpu().numpy()
         check(got, oracle.fake_quantize(rotated(x[torch.as_tensor(rows)].contiguous(), 32), fmt))
     assert bro.last_device_status() == 0
