@@ -585,7 +585,7 @@ def block_sweep(bro, synth, peaks, blocks, groups):
     producer["speedup"] = round(producer["two_step"]["us"] / producer["fused"]["us"], 3)
     del gates, ups, h
     # Simulated quantisation (Sec. 3.1: how the paper evaluates the formats): rotate, quantise, dequantise
-    # to fp32 in one launch — 2 B read and 4 B written per element.
+    # to fp32 in one launch — 2 B read and 4 B written per element (2 + 2 read for the per-row formats).
     deq = torch.empty((M, K), dtype=torch.float32, device="cuda")
     fws = torch.empty(bro.fake_quantize_workspace_bytes(M, "int4_row_asym"), dtype=torch.uint8, device="cuda")
     fake = {}
@@ -602,8 +602,9 @@ def block_sweep(bro, synth, peaks, blocks, groups):
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(c) / ring)
         ms = statistics.mean(ts)
-        fake[fmt] = {"us": round(ms * 1e3, 2), "gbs": round(M * K * 6.0 / (ms * 1e-3) / 1e9, 1),
-                     "frac_of_measured_copy": round(M * K * 6.0 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+        nbytes = 8.0 if fmt.startswith("int4_row") else 6.0      # (the per-row formats read x twice)
+        fake[fmt] = {"us": round(ms * 1e3, 2), "gbs": round(M * K * nbytes / (ms * 1e-3) / 1e9, 1),
+                     "frac_of_measured_copy": round(M * K * nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
     del deq, fws
     return {"shape_MK": [M, K], "algorithmic_bytes": bytes_per_launch, "per_block": per_block,
             "swiglu_producer_block32": producer, "fake_quantize_block32": fake,
