@@ -284,12 +284,13 @@ bro_status bro_rotate_fake_quantize(const void* x_bf16, int64_t M, int64_t K, in
                                     const void* signs_bf16, bro_format format, float* deq, int64_t ldd,
                                     void* stream);
 /*
- * The same with a workspace, which opens three more values of `format`:
+ * The same with a workspace.  Three more values of `format` exist for these two calls (BRO_FMT_NONE
+ * needs no workspace and is accepted by both; the per-row formats need one):
  *   BRO_FMT_INT4_ROW_SYM   INT4 with one scale per ROW, symmetric: |k| <= 7, scale fp16(amax_row / 7)
  *   BRO_FMT_INT4_ROW_ASYM  INT4 with one scale per row, asymmetric: codes q in [0, 15] over the range
  *                          [lo, hi] = [min(row, 0), max(row, 0)], scale s = fp16((hi - lo) / 15), zero
  *                          point z = rint(-lo / s) (at most 15), q = clamp(rint(y / s) + z, 0, 15),
- *                          dequantised (q - z) s
+ *                          dequantised (q - z) s (+0.0 where q == z)
  *   BRO_FMT_NONE           no quantisation: deq = x diag(s) R_block itself, the fp32 values every other
  *                          format is an approximation of (so that the caller can form any error statistic)
  * The first two are the fifth format of the paper's study (Sec. 3.2 / Fig. 2: "INT4" = per-channel
