@@ -172,6 +172,24 @@ class ClockSampler:
     def mark(self, name):
         self.marks[name] = time.time()
 
+    def window(self, t0, t1):
+        """Median SM clock, highest power reading and throttle reasons of the samples taken in [t0, t1]."""
+        sm, power, reasons = [], [], set()
+        for (t, line) in list(self.rows):
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9 or not (t0 <= t <= t1):
+                continue
+            try:
+                sm.append(float(f[1]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "power_w_max": max(power) if power else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -407,7 +425,7 @@ def time_kernels(layers, groups):
     return rq_t, gemm_t
 
 
-def operand_data_effect(layers, i, groups=6):
+def operand_data_effect(layers, i, groups=6, sampler=None):
     """The same GEMM launch timed on the real quantised operands and on operands whose codes are all
     zero (scales, shapes, kernel and launch unchanged).  The instruction stream is identical; what
     differs is how much the tensor pipe's inputs toggle, and with that the power the chip draws and the
@@ -433,6 +451,7 @@ def operand_data_effect(layers, i, groups=6):
         e1.record()
         torch.cuda.synchronize()
         settle = int(min(2000, max(4, 0.3 / max(e0.elapsed_time(e1) * 1e-3 / len(sets), 1e-6))))
+        t_begin = time.time()
         for n in range(settle):
             ac, asc, wc, wsc, y, gws = sets[n % len(sets)]
             bro.gemm_mxfp4(ac, asc, wc, wsc, M, N, K, y, workspace=gws)
@@ -445,12 +464,16 @@ def operand_data_effect(layers, i, groups=6):
             e1.record()
             times.append((e0, e1))
         torch.cuda.synchronize()
-        return statistics.mean(a.elapsed_time(b) for a, b in times) / len(sets) * 1e3
+        t_end = time.time()
+        # what nvidia-smi saw during the run (its first 0.1 s, the transition, left out)
+        seen = sampler.window(t_begin + 0.1, t_end) if sampler is not None and sampler.proc is not None else None
+        return statistics.mean(a.elapsed_time(b) for a, b in times) / len(sets) * 1e3, seen
 
-    us_zero, us_real = run(zero), run(real)
+    (us_zero, seen_zero), (us_real, seen_real) = run(zero), run(real)
     return {"MKN": [M, K, N], "gemm_kernel": gemm_kernel_name(M, K, N), "us_real_operands": round(us_real, 2),
             "us_zero_codes": round(us_zero, 2), "ratio": round(us_real / us_zero, 4),
             "tflops_zero_codes": round(2.0 * M * K * N / us_zero / 1e6, 1),
+            "nvidia_smi_real_operands": seen_real, "nvidia_smi_zero_codes": seen_zero,
             "timing": "each after 0.3 s of back-to-back launches on the same operands",
             "note": "same kernel, launch and instruction stream; all-zero codes draw less power and keep the SM clock "
                     "up, so the ratio is what the chip's power management adds to a sustained run on real operands"}
@@ -681,7 +704,8 @@ def run_ours(args):
         tensor_bound = [i for i, sh in enumerate(shapes) if list(sh) in roofline["shapes"]]
         mid = [i for i in tensor_bound if shapes[i][0] <= 8192] or tensor_bound
         pick = max(mid, key=lambda i: shapes[i][0] * shapes[i][1] * shapes[i][2])
-        roofline["operand_data_effect"] = guarded("operand_data_effect", lambda: operand_data_effect(layers, pick))
+        roofline["operand_data_effect"] = guarded("operand_data_effect",
+                                                  lambda: operand_data_effect(layers, pick, sampler=sampler))
 
     def measure_e2e():
         host = []
